@@ -1,0 +1,173 @@
+"""Pins for the oracle's segment semantics (export / import of ownership segments).
+
+The cipher itself is pinned in test_oracle_crypto.py; here every segment result is
+re-derived with OpenSSL on bytes gathered by the test, and the status / fallback rules
+are checked against hand-built cases.
+"""
+import numpy as np
+from cryptography.hazmat.primitives.ciphers.aead import AESGCM
+
+from oracle import gcm
+from paper_2608_25431_b200 import workloads as W
+
+
+def _gather(w, buf, i):
+    s = w.segs[i]
+    n = int(s["len"])
+    if w.page_table is None:
+        o = int(s["offset"])
+        return buf[o: o + n].tobytes()
+    out = bytearray()
+    pb = w.page_bytes
+    for k in range(0, n, pb):
+        page = int(w.page_table[int(s["page0"]) + k // pb])
+        out += buf[page * pb: page * pb + min(pb, n - k)].tobytes()
+    return bytes(out)
+
+
+def _enc(w, src, dst, **kw):
+    return gcm.seg_encrypt(src, dst, kw.pop("segs", w.segs), w.user_ids, kw.pop("keys", w.keys),
+                           w.max_users, w.page_table, w.page_bytes,
+                           kw.pop("owner_map", w.owner_map), w.unit_bytes)
+
+
+def _check_against_openssl(w, ct, tags, idx):
+    for i in idx:
+        s = w.segs[i]
+        ref = AESGCM(w.keys[int(s["owner"])].tobytes()).encrypt(s["nonce"].tobytes(), _gather(w, w.buf, i), None)
+        assert _gather(w, ct, i) + tags[i].tobytes() == ref, i
+
+
+def test_flat_segments_match_openssl_and_round_trip():
+    w = W.config1()
+    ct = w.buf.copy()
+    tags, st = _enc(w, w.buf, ct)
+    assert not st.any()
+    _check_against_openssl(w, ct, tags, range(len(w.segs)))
+    pt = ct.copy()
+    st = gcm.seg_decrypt(ct, pt, w.segs, tags, w.user_ids, w.keys, w.max_users)
+    assert not st.any() and np.array_equal(pt, w.buf)
+
+
+def test_partial_last_block_rows():
+    w = W.config2(n_users=6, vocab=100)
+    ct = w.buf.copy()
+    tags, st = _enc(w, w.buf, ct)
+    assert not st.any()
+    _check_against_openssl(w, ct, tags, range(6))
+    rows_pt = w.buf.reshape(6, -1)
+    rows_ct = ct.reshape(6, -1)
+    assert np.array_equal(rows_pt[:, 204:], rows_ct[:, 204:])      # pad bytes outside segments untouched
+
+
+def test_paged_segments_match_openssl_in_place():
+    w = W.config4(total_bytes=3 << 20, cap_bytes=1 << 20, n_users=16)
+    ct = w.buf.copy()
+    tags, st = _enc(w, ct, ct)                                     # in place
+    assert not st.any()
+    big = np.argsort(w.segs["len"])[-3:]
+    some = np.random.default_rng(0).choice(len(w.segs), size=min(20, len(w.segs)), replace=False)
+    _check_against_openssl(w, ct, tags, list(big) + list(some))
+    st = gcm.seg_decrypt(ct, ct, w.segs, tags, w.user_ids, w.keys, w.max_users, w.page_table, w.page_bytes)
+    assert not st.any() and np.array_equal(ct, w.buf)
+
+
+def test_table_order_is_irrelevant():
+    w = W.config1()
+    ct = w.buf.copy()
+    tags, _ = _enc(w, w.buf, ct)
+    perm = np.random.default_rng(1).permutation(len(w.segs))
+    ct2 = w.buf.copy()
+    tags2, _ = _enc(w, w.buf, ct2, segs=w.segs[perm])
+    assert np.array_equal(ct, ct2) and np.array_equal(tags[perm], tags2)
+
+
+def test_changing_one_users_key_touches_only_that_user():
+    w = W.config1()
+    ct = w.buf.copy()
+    tags, _ = _enc(w, w.buf, ct)
+    keys2 = w.keys.copy()
+    keys2[3] ^= 0x5A
+    ct2 = w.buf.copy()
+    tags2, _ = _enc(w, w.buf, ct2, keys=keys2)
+    for i, s in enumerate(w.segs):
+        o, n = int(s["offset"]), int(s["len"])
+        same = np.array_equal(ct[o:o + n], ct2[o:o + n]) and np.array_equal(tags[i], tags2[i])
+        assert same == (int(s["owner"]) != 3)
+
+
+def test_export_status_rules():
+    w = W.config2(n_users=8, vocab=64)
+    ST = gcm
+    om = w.owner_map.copy()
+    om[1] = 5                   # another user's label on row 1
+    om[2] = gcm.OWNER_NONE      # unowned
+    om[3] = gcm.OWNER_PARAM     # parameters can never be exported
+    om[4] = gcm.OWNER_CONFLICT
+    segs = w.segs.copy()
+    segs["offset"][5] += 8      # misaligned
+    segs["len"][6] = w.buf.size # out of range
+    ids, keys = w.user_ids[:7], w.keys[:7]          # user 7 has no key
+    dst = np.full_like(w.buf, 0xEE)
+    tags, st = gcm.seg_encrypt(w.buf, dst, segs, ids, keys, w.max_users, None, 0, om, w.unit_bytes)
+    assert st.tolist() == [0, ST.ST_OWNER_MISMATCH, ST.ST_UNOWNED, ST.ST_OWNER_MISMATCH, ST.ST_UNOWNED,
+                           ST.ST_BAD_DESC, ST.ST_BAD_DESC, ST.ST_NO_KEY]
+    rows = dst.reshape(8, -1)
+    assert (rows[1:] == 0xEE).all() and not tags[1:].any()          # failed: bytes as they were, zero tag
+    assert (rows[0, int(segs["len"][0]):] == 0xEE).all() and tags[0].any()
+    # a claimed owner that disagrees with a uniform map is a mismatch too
+    segs = w.segs.copy()
+    segs["owner"][0] = 1
+    _, st = gcm.seg_encrypt(w.buf, dst, segs, w.user_ids, w.keys, w.max_users, None, 0, w.owner_map, w.unit_bytes)
+    assert st[0] == ST.ST_OWNER_MISMATCH and not st[1:].any()
+
+
+def test_import_failure_zero_fills_and_unowns():
+    w = W.config2(n_users=6, vocab=64)
+    ct = w.buf.copy()
+    tags, _ = _enc(w, w.buf, ct)
+    bad_ct = ct.copy()
+    bad_ct[int(w.segs["offset"][1]) + 17] ^= 0x04                   # flipped ciphertext bit
+    bad_tags = tags.copy()
+    bad_tags[2, 9] ^= 0x80                                           # flipped tag bit
+    segs = w.segs.copy()
+    segs["owner"][3] = 0                                             # claims another user's key
+    om = np.full(6, 99, dtype=np.int32)
+    out = np.full_like(ct, 0xEE)
+    st = gcm.seg_decrypt(bad_ct, out, segs, bad_tags, w.user_ids, w.keys, w.max_users,
+                         owner_map=om, unit_bytes=w.unit_bytes)
+    assert st.tolist() == [0, 1, 1, 1, 0, 0]
+    rows, ref = out.reshape(6, -1), w.buf.reshape(6, -1)
+    n = int(w.segs["len"][0])
+    for i in range(6):
+        if st[i]:
+            assert not rows[i, :n].any()
+        else:
+            assert np.array_equal(rows[i, :n], ref[i, :n])
+        assert (rows[i, n:] == 0xEE).all()
+    assert om.tolist() == [0, gcm.OWNER_NONE, gcm.OWNER_NONE, gcm.OWNER_NONE, 4, 5]
+    # verify-only: same statuses, nothing written
+    out2 = np.full_like(ct, 0xEE)
+    om2 = np.full(6, 99, dtype=np.int32)
+    st2 = gcm.seg_decrypt(bad_ct, out2, segs, bad_tags, w.user_ids, w.keys, w.max_users,
+                          owner_map=om2, unit_bytes=w.unit_bytes, verify_only=True)
+    assert st2.tolist() == st.tolist() and (out2 == 0xEE).all() and (om2 == 99).all()
+
+
+def test_empty_segment_tag_is_encrypted_j0():
+    w = W.config1()
+    segs = w.segs[:1].copy()
+    segs["len"] = 0
+    tags, st = gcm.seg_encrypt(w.buf, w.buf.copy(), segs, w.user_ids, w.keys, w.max_users)
+    j0 = segs["nonce"][0].tobytes() + b"\x00\x00\x00\x01"
+    assert st[0] == 0 and tags[0].tobytes() == gcm.aes128_encrypt_block(w.keys[0], j0)
+
+
+def test_workload_generators_are_seeded():
+    a, b = W.config4(total_bytes=1 << 20, cap_bytes=1 << 18, n_users=8), W.config4(total_bytes=1 << 20, cap_bytes=1 << 18, n_users=8)
+    assert np.array_equal(a.buf, b.buf) and np.array_equal(a.segs, b.segs)
+    w5 = W.config5(layers=1, n_users=8, chunk_tokens=4, fill=False)
+    assert len(w5.segs) == 8 and w5.buf_bytes == 20 * W.KV_TOKEN_BYTES
+    w3 = W.config3(layers=1, n_users=2, min_len=17, max_len=40, fill=True)
+    assert w3.buf.size == len(w3.segs) * W.KV_PAGE_BYTES
+    assert sorted(w3.page_table.tolist()) == list(range(len(w3.segs)))
