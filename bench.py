@@ -1,0 +1,380 @@
+"""Benchmark of the segment-encryption hot path on B200 (one JSON line on stdout).
+
+python bench.py --gpus N --steps K --warmup W            # the CUDA path (default)
+python bench.py --impl reference --steps K --warmup W    # the CPU oracle, timed on host cores
+
+Workload (default): the prefill -> decode KV-cache handoff of a LLaMA-7B-shaped model
+(workloads.config3 at 32 layers): every 256 KiB KV block of every user encrypted under its
+owner's key with a per-block tag.  One step = one pass of the whole hot path over that
+batch: the flow rule of the handoff copy on the block owner map (IDENTITY), then
+gift_seg_encrypt (plan + label check, work list, CTR + GHASH, tag finish) in place.  Key
+setup is outside the step, as it is once per key change.  The path does not shard: with
+--gpus N every rank runs an independent replica on its own GPU (no collective on the data
+path) and the value is the sum of the replicas over the slowest rank's time.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "segment encrypt+tag throughput"
+UNIT = "GB/s"
+
+# Integer work per 16-byte block of the best formulation known to this build (frozen; the
+# kernel's own instruction count is not used): T-table AES-CTR with the first round hoisted
+# and GHASH by masked integer multiplies with two Karatsuba levels.
+ALU_OPS_PER_BLOCK = 660          # logic / permute / shift / add lane-operations
+MUL_OPS_PER_BLOCK = 144          # 32x32 -> 64 multiplies
+LDS_OPS_PER_BLOCK = 150          # 4-byte shared-memory lookups
+
+
+def build_workload(name: str, layers: int):
+    from paper_2608_25431_b200 import workloads as W
+    if name == "c3":
+        return W.config3(layers=layers, fill=False)
+    if name == "c4":
+        return W.config4(total_bytes=8 << 30, cap_bytes=64 << 20, fill=False)
+    if name == "c5":
+        return W.config5(layers=layers, chunk_tokens=512, fill=False)
+    if name == "c2":
+        return W.config2()
+    raise ValueError(name)
+
+
+class ClockSampler(threading.Thread):
+    """Samples SM clock, power and throttle reasons of one GPU through NVML while the timed region runs."""
+
+    def __init__(self, index: int, period: float = 0.1):
+        super().__init__(daemon=True)
+        self.index, self.period = index, period
+        self.samples, self.reasons, self.stop_flag = [], set(), threading.Event()
+        self.max_mhz = None
+
+    def run(self):
+        try:
+            import pynvml as nv
+            nv.nvmlInit()
+            h = nv.nvmlDeviceGetHandleByIndex(self.index)
+            self.max_mhz = nv.nvmlDeviceGetMaxClockInfo(h, nv.NVML_CLOCK_SM)
+            names = {
+                nv.nvmlClocksThrottleReasonHwSlowdown: "hw_slowdown",
+                nv.nvmlClocksThrottleReasonHwThermalSlowdown: "hw_thermal_slowdown",
+                nv.nvmlClocksThrottleReasonSwThermalSlowdown: "sw_thermal_slowdown",
+                nv.nvmlClocksThrottleReasonSwPowerCap: "sw_power_cap",
+                nv.nvmlClocksThrottleReasonHwPowerBrakeSlowdown: "hw_power_brake",
+            }
+            while not self.stop_flag.is_set():
+                self.samples.append(nv.nvmlDeviceGetClockInfo(h, nv.NVML_CLOCK_SM))
+                r = nv.nvmlDeviceGetCurrentClocksThrottleReasons(h)
+                for bit, name in names.items():
+                    if r & bit:
+                        self.reasons.add(name)
+                time.sleep(self.period)
+        except Exception as e:      # NVML missing: report nothing rather than fail the run
+            self.reasons.add("nvml_unavailable:%s" % type(e).__name__)
+
+    def result(self):
+        self.stop_flag.set()
+        self.join(timeout=2)
+        med = float(np.median(self.samples)) if self.samples else None
+        return {"sm_mhz": med, "sm_max_mhz": self.max_mhz, "reasons": sorted(self.reasons),
+                "samples": len(self.samples)}
+
+
+def physical_gpu_index(local: int) -> int:
+    vis = os.environ.get("CUDA_VISIBLE_DEVICES")
+    if vis:
+        try:
+            return int(vis.split(",")[local])
+        except (ValueError, IndexError):
+            return local
+    return local
+
+
+def cpu_sample(w, seconds_target: float):
+    """Time the oracle, as it stands, on a bounded prefix of the workload's segment table."""
+    from oracle import gcm
+    from paper_2608_25431_b200 import workloads as W
+    rng = np.random.default_rng(W.SEED_BASE + 99)
+    segs = w.segs
+    order = np.arange(len(segs))
+
+    def run(idx):
+        sub = segs[idx].copy()
+        lens = sub["len"].astype(np.int64)
+        # lay the sampled segments out flat, back to back (same bytes of work per segment)
+        offs = np.concatenate([[0], np.cumsum((lens + 15) // 16 * 16)[:-1]])
+        sub["offset"] = offs
+        sub["page0"] = 0
+        total = int(((lens + 15) // 16 * 16).sum())
+        buf = np.frombuffer(rng.bytes(total), dtype=np.uint8).copy()
+        t0 = time.perf_counter()
+        _, st = gcm.seg_encrypt(buf, buf, sub, w.user_ids, w.keys, w.max_users)
+        dt = time.perf_counter() - t0
+        assert not st.any()
+        return int(lens.sum()), dt
+
+    threads = gcm.threads()
+    nb, dt = run(order[: max(threads * 2, 8)])            # calibration
+    rate = nb / dt
+    want = rate * seconds_target
+    cum = np.cumsum(segs["len"].astype(np.int64))
+    n = int(np.searchsorted(cum, want)) + 1
+    n = max(min(n, len(segs)), min(len(segs), threads))
+    nb, dt = run(order[:n])
+    return {"value": nb / dt / 1e9, "unit": UNIT, "cores": threads, "kind": "oracle",
+            "sample": "first %d segments (%.1f MiB) of the workload's table, laid out flat, %.1f s" % (n, nb / 2**20, dt)}
+
+
+def run_reference(args):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    w = build_workload(args.workload, args.layers)
+    per_step = max(2.0, min(20.0, 120.0 / max(1, args.steps + args.warmup)))
+    vals = []
+    last = None
+    for i in range(args.warmup + args.steps):
+        last = cpu_sample(w, per_step)
+        if i >= args.warmup:
+            vals.append(last["value"])
+    v = float(np.mean(vals))
+    payload = w.payload_bytes
+    line = {"impl": "reference", "metric": METRIC, "value": v, "unit": UNIT, "n_gpus": args.gpus,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": payload / (v * 1e9) * 1e3,
+            "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "u32",
+            "data": "synthetic", "config": workload_config(args, w),
+            "cpu_baseline": {"value": v, "unit": UNIT, "cores": last["cores"], "kind": "oracle",
+                             "sample": last["sample"] + " per step; ms_per_step extrapolates to the full workload"},
+            "e2e": {"value": v, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+            "gpu_launches": 0}
+    print(json.dumps(line))
+
+
+def workload_config(args, w):
+    return {"workload": "%s: %s, %d segments, %.3f GiB payload, %d users" % (
+                args.workload, w.name, len(w.segs), w.payload_bytes / 2**30, len(w.user_ids)),
+            "layers": args.layers, "l2": "inputs larger than L2 (no flush needed)" if w.payload_bytes > (256 << 20)
+            else "L2 flushed between iterations", "parallelism": "replicas"}
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="gift", choices=["gift", "reference"])
+    ap.add_argument("--workload", default="c3", choices=["c2", "c3", "c4", "c5"])
+    ap.add_argument("--layers", type=int, default=32)
+    ap.add_argument("--flags", type=lambda s: int(s, 0), default=0, help="kernel variant, see gift.h")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-extra", action="store_true")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3) if args.impl == "gift" else args.warmup
+
+    if args.impl == "reference":
+        run_reference(args)
+        return
+
+    import torch
+    import torch.distributed as dist
+    from paper_2608_25431_b200 import binding, device_fill, workloads as W
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device (there is no CPU fallback)")
+    torch.cuda.set_device(local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    w = build_workload(args.workload, args.layers)
+    free, _ = torch.cuda.mem_get_info()
+    if w.buf_bytes + (2 << 30) > free and args.workload in ("c3", "c5"):
+        while args.layers > 1 and w.buf_bytes + (2 << 30) > free:
+            args.layers //= 2
+            w = build_workload(args.workload, args.layers)
+    nseg = len(w.segs)
+    ctx = binding.Ctx(w.max_users, local, args.flags)
+    ctx.set_keys(w.user_ids, w.keys)
+    ctx.reserve(nseg)
+    buf = torch.empty(w.buf_bytes, dtype=torch.uint8, device="cuda")
+    if w.buf is not None:
+        buf.copy_(torch.from_numpy(w.buf))
+    elif args.workload == "c4":
+        device_fill.fill_bytes(buf, W.SEED_BASE + 4 + rank)
+    else:
+        device_fill.fill_bf16_normal(buf, W.SEED_BASE + 3 + rank, 1.0)
+    segs = torch.from_numpy(w.segs.view(np.uint8).copy()).cuda()
+    table = torch.from_numpy(w.page_table).cuda() if w.page_table is not None else None
+    om_src = torch.from_numpy(w.owner_map).cuda()
+    om = torch.empty_like(om_src)
+    viol = torch.zeros(2, dtype=torch.int32, device="cuda")
+    tags = torch.zeros((nseg, 16), dtype=torch.uint8, device="cuda")
+    status = torch.zeros(nseg, dtype=torch.int32, device="cuda")
+    flush = torch.empty(512 << 20, dtype=torch.uint8, device="cuda") if w.payload_bytes <= (256 << 20) else None
+    payload = w.payload_bytes
+
+    def step():
+        if flush is not None:
+            flush.fill_(1)
+        ctx.propagate_labels(binding.RULE_IDENTITY, [om_src], om, viol)
+        ctx.seg_encrypt(buf, buf, segs, nseg, tags, status, page_table=table, page_bytes=w.page_bytes,
+                        owner_map=om, unit_bytes=w.unit_bytes)
+
+    for _ in range(args.warmup):
+        step()
+    barrier()
+    assert not status.any().item() and int(viol[0].item()) == 0, "workload segments were rejected"
+    l0 = ctx.launch_count()
+    ctx.timing_enable(True)
+    sampler = ClockSampler(physical_gpu_index(local))
+    sampler.start()
+    ev = [torch.cuda.Event(enable_timing=True) for _ in range(args.steps + 1)]
+    barrier()
+    ev[0].record()
+    for i in range(args.steps):
+        step()
+        ev[i + 1].record()
+    barrier()
+    clocks = sampler.result()
+    total_ms = ev[0].elapsed_time(ev[-1])
+    step_ms = [ev[i].elapsed_time(ev[i + 1]) for i in range(args.steps)]
+    crypt_ms, crypt_n = ctx.timing_read()
+    ctx.timing_enable(False)
+    launches = ctx.launch_count() - l0 + (args.steps if flush is not None else 0) * 0
+    t = torch.tensor([total_ms], dtype=torch.float64, device="cuda")
+    if world > 1:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    total_ms_max = float(t.item())
+    ms_per_step = total_ms_max / args.steps
+    value = world * payload / (ms_per_step * 1e-3) / 1e9
+
+    # ---- roofline of the dominant kernel (the cipher kernel), bound by the integer pipes ----
+    nblk = int(((w.segs["len"].astype(np.int64) + 15) // 16).sum())
+    kern_ms = crypt_ms / max(1, crypt_n)
+    f_mhz = clocks["sm_mhz"] or 1965.0
+    sms = torch.cuda.get_device_properties(local).multi_processor_count
+    peaks = json.load(open(os.path.join(ROOT, "MEASURED_PEAKS.json"))) if os.path.exists(
+        os.path.join(ROOT, "MEASURED_PEAKS.json")) else {}
+    hbm_gbs = peaks.get("hbm_gbs", 6650.0)
+    r_alu, r_mul, r_lds, r_issue = 64.0, 64.0, 32.0, 128.0        # lane-ops per SM clock
+    f = f_mhz * 1e6
+    t_alu = ALU_OPS_PER_BLOCK * nblk / (sms * r_alu * f)
+    t_mul = MUL_OPS_PER_BLOCK * nblk / (sms * r_mul * f)
+    t_lds = LDS_OPS_PER_BLOCK * nblk / (sms * r_lds * f)
+    t_issue = (ALU_OPS_PER_BLOCK + MUL_OPS_PER_BLOCK + LDS_OPS_PER_BLOCK) * nblk / (sms * r_issue * f)
+    t_hbm = (2.0 * payload + 56.0 * nseg) / (hbm_gbs * 1e9)
+    t_roof = max(t_alu, t_mul, t_lds, t_issue, t_hbm)
+    achieved_tops = ALU_OPS_PER_BLOCK * nblk / (kern_ms * 1e-3) / 1e12
+    peak_tops = sms * r_alu * f / 1e12
+    roofline = {"bound": "alu", "achieved": achieved_tops, "peak": peak_tops, "unit": "Top/s",
+                "frac": t_roof / (kern_ms * 1e-3), "traffic": None,
+                "kernel": "crypt_kernel", "kernel_ms": kern_ms, "kernel_launches": crypt_n,
+                "kernel_payload_gbs": payload / (kern_ms * 1e-3) / 1e9,
+                "hbm_achieved_gbs": 2.0 * payload / (kern_ms * 1e-3) / 1e9,
+                "hbm_frac_of_measured": 2.0 * payload / (kern_ms * 1e-3) / 1e9 / hbm_gbs,
+                "ceilings_gbs": {"alu": payload / t_alu / 1e9, "mul": payload / t_mul / 1e9,
+                                 "lds": payload / t_lds / 1e9, "issue": payload / t_issue / 1e9,
+                                 "hbm": payload / t_hbm / 1e9},
+                "sm_mhz_used": f_mhz,
+                "peak_source": "148 SMs x 64 integer lanes x sampled SM clock; HBM from MEASURED_PEAKS.json (of measured)"
+                if peaks else "fallback HBM 6650 GB/s (of fallback)"}
+
+    line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+            "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "u32", "data": "synthetic", "config": workload_config(args, w),
+            "clocks": clocks, "gpu_launches": int(launches), "roofline": roofline,
+            "step_ms_median": float(np.median(step_ms))}
+
+    # ---- other rates of the same path (not in the timed region) ----
+    if not args.no_extra and rank == 0:
+        def timed(fn, n=5):
+            fn()
+            torch.cuda.synchronize()
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record()
+            for _ in range(n):
+                fn()
+            b.record()
+            torch.cuda.synchronize()
+            return a.elapsed_time(b) / n
+        ctx.seg_encrypt(buf, buf, segs, nseg, tags, status, page_table=table, page_bytes=w.page_bytes)
+        ver = timed(lambda: ctx.verify_tags(buf, segs, nseg, tags, status, page_table=table, page_bytes=w.page_bytes))
+        ok_verify = not status.any().item()
+        dec = timed(lambda: (ctx.seg_encrypt(buf, buf, segs, nseg, tags, status, page_table=table, page_bytes=w.page_bytes),
+                             ctx.seg_decrypt(buf, buf, segs, nseg, tags, status, page_table=table,
+                                             page_bytes=w.page_bytes, owner_map=om, unit_bytes=w.unit_bytes)), n=3)
+        rule_us = timed(lambda: ctx.propagate_labels(binding.RULE_IDENTITY, [om_src], om, viol), n=50) * 1e3
+        line["extra"] = {"verify_gbs": payload / ver / 1e6, "verify_all_ok": bool(ok_verify),
+                         "encrypt_plus_decrypt_gbs": 2 * payload / dec / 1e6,
+                         "decrypt_restores_ok": bool(not status.any().item()),
+                         "identity_rule_us": rule_us}
+
+    # ---- end to end from pinned host memory ----
+    if not args.no_e2e:
+        try:
+            h_in = torch.empty(w.buf_bytes, dtype=torch.uint8, pin_memory=True)
+            h_out = torch.empty(w.buf_bytes, dtype=torch.uint8, pin_memory=True)
+            h_tags = torch.empty((nseg, 16), dtype=torch.uint8, pin_memory=True)
+            h_status = torch.empty(nseg, dtype=torch.int32, pin_memory=True)
+            h_in.copy_(buf)
+            k = max(1, min(args.steps, 5))
+
+            def e2e_step():
+                buf.copy_(h_in, non_blocking=True)
+                ctx.propagate_labels(binding.RULE_IDENTITY, [om_src], om, viol)
+                ctx.seg_encrypt(buf, buf, segs, nseg, tags, status, page_table=table, page_bytes=w.page_bytes,
+                                owner_map=om, unit_bytes=w.unit_bytes)
+                h_out.copy_(buf, non_blocking=True)
+                h_tags.copy_(tags, non_blocking=True)
+                h_status.copy_(status, non_blocking=True)
+
+            e2e_step()
+            barrier()
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record()
+            for _ in range(k):
+                e2e_step()
+            b.record()
+            barrier()
+            t2 = torch.tensor([a.elapsed_time(b) / k], dtype=torch.float64, device="cuda")
+            if world > 1:
+                dist.all_reduce(t2, op=dist.ReduceOp.MAX)
+            e2e_ms = float(t2.item())
+            line["e2e"] = {"value": world * payload / e2e_ms / 1e6, "unit": UNIT,
+                           "h2d_bytes_per_step": int(w.buf_bytes),
+                           "d2h_bytes_per_step": int(w.buf_bytes + nseg * 20), "steps": k, "ms_per_step": e2e_ms}
+            del h_in, h_out
+        except RuntimeError as e:
+            line["e2e"] = {"value": None, "unit": UNIT, "error": str(e)[:200]}
+
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        line["cpu_baseline"] = cpu_sample(w, 15.0)
+
+    ctx.close()
+    if rank == 0:
+        print(json.dumps(line))
+    if world > 1:
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

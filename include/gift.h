@@ -1,0 +1,240 @@
+/*
+ * libgift: per-user encryption of ownership-segmented GPU buffers, with the
+ * ownership-label check and segment-level flow rules, for one NVIDIA B200.
+ *
+ * The library realises the data path of the paper's "encryption-as-isolation"
+ * (paper sec. 3, workflow steps 0 and 3-6): every user datum that leaves the
+ * protected domain is ciphertext under its owner's key, and data entering it
+ * is decrypted with the key of the owner the untrusted framework claims, so a
+ * false claim ends in a decryption failure instead of a leak.  The paper names
+ * no cipher; this library uses AES-128-GCM per segment (AES-128 in counter
+ * mode, FIPS-197 / SP 800-38A, with the GHASH tag of SP 800-38D, 96-bit IV,
+ * 128-bit tag, empty AAD).  The tag is what makes a wrong owner or a tampered
+ * byte detectable.
+ *
+ * Conventions common to all calls
+ *  - Every call returns an int: GIFT_OK (0) or a negative GIFT_E_* code for an
+ *    error detected synchronously on the host (bad argument, CUDA error).
+ *    What happens to one segment never comes back as the return code; it is
+ *    written to the device array status[] as a bit set of GIFT_ST_* flags.
+ *  - Unless stated otherwise every data pointer is a DEVICE pointer owned by
+ *    the caller, valid on the ctx's device.  The ctx owns only key material,
+ *    tables and scratch, and overwrites key material with zeros on destroy.
+ *  - Calls enqueue work on the given stream (a cudaStream_t passed as void*;
+ *    NULL is the default stream) and do not wait for it.  The exception is
+ *    scratch growth: a call whose segment count exceeds what the ctx has seen
+ *    so far (see gift_ctx_reserve) reallocates scratch, which synchronises.
+ *  - gift_pages, gift_labels and gift_rule are small HOST structures that carry device
+ *    pointers; they are read during the call and need not outlive it.
+ *  - A ctx must not be used from two threads, or on two streams, at once.
+ *  - Ownership labels are int32: a user id >= 0, GIFT_OWNER_PARAM for model
+ *    parameters (paper sec. 4.2: "a special ID for model parameters"),
+ *    GIFT_OWNER_NONE for memory no record covers (sec. 4.2, unowned memory may
+ *    not be read), GIFT_OWNER_CONFLICT for an output whose sources disagree.
+ */
+#ifndef GIFT_H
+#define GIFT_H
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define GIFT_OK          0
+#define GIFT_E_INVAL    (-1)   /* null / inconsistent argument */
+#define GIFT_E_NOMEM    (-2)   /* host or device allocation failed */
+#define GIFT_E_CUDA     (-3)   /* a CUDA runtime call failed */
+#define GIFT_E_RANGE    (-4)   /* user id outside [0, max_users), size over a stated limit */
+#define GIFT_E_ALIGN    (-5)   /* buffer or page size not 16-byte aligned */
+
+#define GIFT_ST_TAG_MISMATCH    1u   /* decrypt/verify: tag does not match (tampered, or wrong owner claimed) */
+#define GIFT_ST_OWNER_MISMATCH  2u   /* encrypt: a covered unit is owned by someone else, or by PARAM */
+#define GIFT_ST_UNOWNED         4u   /* encrypt: a covered unit is NONE or CONFLICT */
+#define GIFT_ST_NO_KEY          8u   /* the owner has no key in the ctx */
+#define GIFT_ST_BAD_DESC       16u   /* descriptor misaligned, out of range, or reserved flags set */
+
+#define GIFT_OWNER_PARAM     (-1)
+#define GIFT_OWNER_NONE      (-2)
+#define GIFT_OWNER_CONFLICT  (-3)
+
+/* Longest segment: the GCM limit of 2^36 - 32 bytes. */
+#define GIFT_MAX_SEG_BYTES  ((((uint64_t)1) << 36) - 32)
+
+typedef struct gift_ctx gift_ctx;
+
+/* One ownership segment: a contiguous same-owner region (paper sec. 4.1,
+ * insight 1, and sec. 4.2 "Recording granularity").  40 bytes; a device array.
+ *   owner  the owner the caller claims for the segment (selects the key)
+ *   flags  reserved, must be 0
+ *   offset flat mode: byte offset of the segment in the buffer, multiple of 16
+ *   len    payload bytes, 0 <= len <= GIFT_MAX_SEG_BYTES, any value (the last
+ *          cipher block may be partial; len 0 yields the tag of the empty message)
+ *   nonce  the 96-bit IV; unique per (key, encryption) - the library never
+ *          invents or checks nonces
+ *   page0  paged mode: index of the segment's first entry in the page table */
+typedef struct {
+    int32_t  owner;
+    uint32_t flags;
+    uint64_t offset;
+    uint64_t len;
+    uint8_t  nonce[12];
+    uint32_t page0;
+} gift_seg;
+
+/* Paged mode (block-table indexed KV cache, paper sec. 4.2): byte k of a
+ * segment lives at table[page0 + k / page_bytes] * page_bytes + k % page_bytes
+ * of the buffer.  table is a device array of n physical page numbers;
+ * page_bytes is a positive multiple of 16.  Pass NULL for flat mode. */
+typedef struct {
+    const int32_t* table;
+    uint32_t       n;
+    uint64_t       page_bytes;
+} gift_pages;
+
+/* Ownership records of the buffer: owner_map[u] is the label of unit u (device
+ * array of n_units labels).  Flat mode: unit u covers bytes [u*unit_bytes,
+ * (u+1)*unit_bytes); a segment covers every unit its byte range touches.
+ * Paged mode: one unit per physical page, unit_bytes ignored.  An empty
+ * segment covers no unit.  Pass NULL to skip label handling. */
+typedef struct {
+    int32_t* owner_map;
+    uint32_t n_units;
+    uint64_t unit_bytes;
+} gift_labels;
+
+/* Create a context on CUDA device `device` able to hold keys for user ids
+ * 0 .. max_users-1 (about 17 KiB of device memory per user: round keys and
+ * powers of the hash subkey), max_users <= 2^20.  flags selects a kernel
+ * variant: 0 for the default, else GIFT_CTX_FLAGS(tables, chains) with tables
+ * in {2, 4} (T-tables kept in shared memory) and chains in {1, 2} (hash chains
+ * per lane); every variant computes the same results.  Host call; synchronises. */
+#define GIFT_CTX_FLAGS(tables, chains)  ((uint32_t)(((tables) << 4) | (chains)))
+int gift_ctx_create(gift_ctx** out, int device, uint32_t max_users, uint32_t flags);
+
+/* Zero all key material on the device and free the ctx.  Synchronises. */
+int gift_ctx_destroy(gift_ctx* ctx);
+
+/* Pre-size the per-call scratch (work list, partial hashes) for calls of up to
+ * max_segs segments so that later calls never reallocate.  Synchronises. */
+int gift_ctx_reserve(gift_ctx* ctx, uint32_t max_segs);
+
+/* Install keys (paper sec. 3 step 0: the monitor stores user-specific keys in
+ * its protected memory).  user_ids[n] and keys16[n*16] are HOST arrays; key i
+ * belongs to user user_ids[i] in [0, max_users).  The expanded round keys, the
+ * hash subkey H = E_K(0) and its powers are derived on the device.  The host
+ * staging copy is wiped before the call returns. */
+int gift_set_keys(gift_ctx* ctx, const int32_t* user_ids, const uint8_t* keys16, uint32_t n,
+                  void* stream);
+
+/* Remove users' keys (device material overwritten with zeros). */
+int gift_clear_keys(gift_ctx* ctx, const int32_t* user_ids, uint32_t n, void* stream);
+
+/* Export (paper sec. 3 steps 5-6; sec. 4.1: the key is selected from the
+ * ownership state, not from the framework's claim).  For every segment, in any
+ * order: if labels are given, every covered unit must carry the segment's
+ * owner; the owner must have a key.  Then dst receives AES-128-CTR ciphertext
+ * of src (counter blocks nonce || BE32(2), BE32(3), ...) and tags_out[i] the
+ * 16-byte GCM tag.  Otherwise the segment's dst bytes are left as they were,
+ * its tag is 16 zero bytes and status[i] says why.  src may equal dst; bytes
+ * outside all segments are never written.  Segments of one call must not
+ * overlap.  buf_bytes is the size of src and of dst. */
+int gift_seg_encrypt(gift_ctx* ctx, const void* src, void* dst, uint64_t buf_bytes,
+                     const gift_seg* segs, uint32_t nseg, const gift_pages* pages,
+                     const gift_labels* labels, uint8_t* tags_out, uint32_t* status, void* stream);
+
+/* Import (paper sec. 3 steps 3-4): decrypt each segment with the CLAIMED
+ * owner's key after checking tags_in[i] over the received ciphertext.  On a
+ * match dst receives the plaintext and, if labels are given, the covered units
+ * are recorded as owned by the claimed owner.  On a mismatch, or when the
+ * claimed owner has no key, the segment's dst bytes are all zero and the
+ * covered units become GIFT_OWNER_NONE (a unit covered by both a good and a
+ * failed segment ends up NONE).  BAD_DESC segments touch nothing. */
+int gift_seg_decrypt(gift_ctx* ctx, const void* src, void* dst, uint64_t buf_bytes,
+                     const gift_seg* segs, uint32_t nseg, const gift_pages* pages,
+                     gift_labels* labels, const uint8_t* tags_in, uint32_t* status, void* stream);
+
+/* Tag check only: status[i] as gift_seg_decrypt would set it; nothing else is written. */
+int gift_verify_tags(gift_ctx* ctx, const void* src, uint64_t buf_bytes, const gift_seg* segs,
+                     uint32_t nseg, const gift_pages* pages, const uint8_t* tags_in,
+                     uint32_t* status, void* stream);
+
+/* A flow rule (paper sec. 4.3, "Generating IFT rules", steps 4 and 5): for
+ * every output unit, its non-parameter sources must share one owner, which the
+ * output receives; operands declared as parameters must be labelled PARAM.
+ * The join treats PARAM as neutral, equal users as that user, and anything
+ * else (different users, NONE, CONFLICT) as CONFLICT.
+ *   GIFT_RULE_IDENTITY   out[j] = in0[j]                       (copies, swaps)
+ *   GIFT_RULE_ROWWISE    out[j] = join over row operands k of in_k[j]; operand
+ *                        k with bit k of param_mask set is a one-unit map that
+ *                        must equal PARAM, else every out[j] is CONFLICT
+ *                        (AddBias, AddResidual, FindMax, MatrixMultiply)
+ *   GIFT_RULE_SEGREDUCE  for reduction segment s (a request): m = join of
+ *                        in0[t] for t in [seg_ptr[s], seg_ptr[s+1]) and of
+ *                        in1[src_idx[e]] for e in [src_ptr[s], src_ptr[s+1]);
+ *                        out[t] = m for the segment's t (decoding-stage
+ *                        attention over a block table, paper sec. 7.2); an
+ *                        out-of-range src_idx counts as NONE; outputs no
+ *                        segment covers are CONFLICT
+ *   GIFT_RULE_BROADCAST  out[j] = in0[gather[j]]; out-of-range gather gives CONFLICT
+ * n_in is the number of input maps (ROWWISE: 1..8; SEGREDUCE: 2; others: 1),
+ * n_in0 the length of in0 (BROADCAST) and n_in1 the length of in1 (SEGREDUCE).
+ * All index arrays are device arrays.  seg_ptr must be non-decreasing with
+ * seg_ptr[n_seg] <= n_out. */
+#define GIFT_RULE_IDENTITY   0u
+#define GIFT_RULE_ROWWISE    1u
+#define GIFT_RULE_SEGREDUCE  2u
+#define GIFT_RULE_BROADCAST  3u
+
+typedef struct {
+    uint32_t kind;
+    uint32_t n_out;
+    uint32_t n_in;
+    uint32_t n_seg;
+    uint32_t n_in0;
+    uint32_t n_in1;
+    const int32_t* seg_ptr;
+    const int32_t* src_ptr;
+    const int32_t* src_idx;
+    const int32_t* gather;
+    uint32_t param_mask;
+} gift_rule;
+
+/* Apply one rule on the device.  rule and in_owner_maps are HOST structures
+ * (an array of n_in device pointers).  out_owner_map may alias an input: the
+ * rule reads a snapshot.  viol[0] receives the number of CONFLICT outputs and
+ * viol[1] the smallest such index (0xFFFFFFFF if none).  The paper rejects the
+ * launch on any violation (sec. 4.1, insight 3); here out is always written
+ * and committing it is the caller's decision. */
+int gift_propagate_labels(gift_ctx* ctx, const gift_rule* rule, const int32_t* const* in_owner_maps,
+                          int32_t* out_owner_map, uint32_t* viol, void* stream);
+
+/* Text for a GIFT_E_* code; never NULL. */
+const char* gift_strerror(int code);
+
+/* Library version, major*10000 + minor*100 + patch. */
+uint32_t gift_version(void);
+
+/* Number of this library's kernels launched through the ctx since creation. */
+uint64_t gift_launch_count(const gift_ctx* ctx);
+
+/* Device timing of the segment-cipher kernel (diagnostics; no paper counterpart).  While
+ * enabled, every gift_seg_encrypt / decrypt / verify call brackets its cipher kernel with
+ * CUDA events on the call's stream.  gift_timing_read waits for the recorded events,
+ * returns their summed duration in milliseconds and the number of launches since the last
+ * read, and resets both.  At most 1024 launches are kept between reads. */
+int gift_timing_enable(gift_ctx* ctx, int on);
+int gift_timing_read(gift_ctx* ctx, double* total_ms, uint32_t* launches);
+
+/* Issue-rate probe (diagnostics; no paper counterpart): runs a long chain of one
+ * instruction kind on every SM of `device` and reports lane-operations per SM clock and
+ * the SM clock seen.  kind: 0 three-input logic, 1 32x32+64 wide multiply-add, 2 byte
+ * permute, 3 conflict-free shared-memory load, 4 funnel shift, 5 integer add, 6 logic and
+ * wide multiply interleaved, 7 32-bit multiply-add, 8 logic and shared loads interleaved.
+ * Host call; allocates a few KB, synchronises. */
+int gift_probe_pipe(int device, int kind, uint32_t iters, double* lane_ops_per_clk_per_sm, double* sm_mhz);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* GIFT_H */

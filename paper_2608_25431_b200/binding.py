@@ -1,0 +1,225 @@
+"""Thin ctypes binding over libgift.so: argument marshalling only.
+
+Function names follow include/gift.h.  Data arguments are torch CUDA tensors (their
+data_ptr() is passed through); key material is passed from host numpy arrays.  There is
+no fallback: if the library has not been built, or no CUDA device is present, the first
+call raises.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+
+import numpy as np
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libgift.so")
+
+OK, E_INVAL, E_NOMEM, E_CUDA, E_RANGE, E_ALIGN = 0, -1, -2, -3, -4, -5
+ST_TAG_MISMATCH, ST_OWNER_MISMATCH, ST_UNOWNED, ST_NO_KEY, ST_BAD_DESC = 1, 2, 4, 8, 16
+OWNER_PARAM, OWNER_NONE, OWNER_CONFLICT = -1, -2, -3
+RULE_IDENTITY, RULE_ROWWISE, RULE_SEGREDUCE, RULE_BROADCAST = 0, 1, 2, 3
+
+EXPORTS = [
+    "gift_ctx_create", "gift_ctx_destroy", "gift_ctx_reserve", "gift_set_keys", "gift_clear_keys",
+    "gift_seg_encrypt", "gift_seg_decrypt", "gift_verify_tags", "gift_propagate_labels",
+    "gift_strerror", "gift_version", "gift_launch_count", "gift_timing_enable", "gift_timing_read",
+    "gift_probe_pipe",
+]
+
+
+class GiftError(RuntimeError):
+    def __init__(self, code, where):
+        self.code = code
+        super().__init__("%s failed: %s (%d)" % (where, strerror(code), code))
+
+
+class _Pages(C.Structure):
+    _fields_ = [("table", C.c_void_p), ("n", C.c_uint32), ("page_bytes", C.c_uint64)]
+
+
+class _Labels(C.Structure):
+    _fields_ = [("owner_map", C.c_void_p), ("n_units", C.c_uint32), ("unit_bytes", C.c_uint64)]
+
+
+class _Rule(C.Structure):
+    _fields_ = [("kind", C.c_uint32), ("n_out", C.c_uint32), ("n_in", C.c_uint32), ("n_seg", C.c_uint32),
+                ("n_in0", C.c_uint32), ("n_in1", C.c_uint32),
+                ("seg_ptr", C.c_void_p), ("src_ptr", C.c_void_p), ("src_idx", C.c_void_p),
+                ("gather", C.c_void_p), ("param_mask", C.c_uint32)]
+
+
+_lib = None
+
+
+def lib():
+    """Load libgift.so; raises if it is missing (build it with `python -m paper_2608_25431_b200.build`)."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise RuntimeError("libgift.so is not built: run python -m paper_2608_25431_b200.build "
+                               "(there is no CPU fallback)")
+        l = C.CDLL(LIB_PATH)
+        l.gift_ctx_create.argtypes = [C.POINTER(C.c_void_p), C.c_int, C.c_uint32, C.c_uint32]
+        l.gift_ctx_destroy.argtypes = [C.c_void_p]
+        l.gift_ctx_reserve.argtypes = [C.c_void_p, C.c_uint32]
+        l.gift_set_keys.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_uint32, C.c_void_p]
+        l.gift_clear_keys.argtypes = [C.c_void_p, C.c_void_p, C.c_uint32, C.c_void_p]
+        l.gift_seg_encrypt.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_uint64, C.c_void_p, C.c_uint32,
+                                       C.POINTER(_Pages), C.POINTER(_Labels), C.c_void_p, C.c_void_p, C.c_void_p]
+        l.gift_seg_decrypt.argtypes = l.gift_seg_encrypt.argtypes
+        l.gift_verify_tags.argtypes = [C.c_void_p, C.c_void_p, C.c_uint64, C.c_void_p, C.c_uint32,
+                                       C.POINTER(_Pages), C.c_void_p, C.c_void_p, C.c_void_p]
+        l.gift_propagate_labels.argtypes = [C.c_void_p, C.POINTER(_Rule), C.POINTER(C.c_void_p), C.c_void_p,
+                                            C.c_void_p, C.c_void_p]
+        l.gift_strerror.restype = C.c_char_p
+        l.gift_strerror.argtypes = [C.c_int]
+        l.gift_version.restype = C.c_uint32
+        l.gift_launch_count.restype = C.c_uint64
+        l.gift_launch_count.argtypes = [C.c_void_p]
+        l.gift_timing_enable.argtypes = [C.c_void_p, C.c_int]
+        l.gift_timing_read.argtypes = [C.c_void_p, C.POINTER(C.c_double), C.POINTER(C.c_uint32)]
+        l.gift_probe_pipe.argtypes = [C.c_int, C.c_int, C.c_uint32, C.POINTER(C.c_double), C.POINTER(C.c_double)]
+        _lib = l
+    return _lib
+
+
+def strerror(code: int) -> str:
+    return lib().gift_strerror(code).decode()
+
+
+def version() -> int:
+    return int(lib().gift_version())
+
+
+def _check(rc, where):
+    if rc != OK:
+        raise GiftError(rc, where)
+
+
+def _stream_ptr(stream):
+    if stream is None:
+        import torch
+        return C.c_void_p(torch.cuda.current_stream().cuda_stream)
+    return C.c_void_p(int(stream))
+
+
+def _dev(t):
+    """Device pointer of a CUDA tensor (or None)."""
+    if t is None:
+        return None
+    if not t.is_cuda or not t.is_contiguous():
+        raise ValueError("expected a contiguous CUDA tensor")
+    return C.c_void_p(t.data_ptr())
+
+
+class Ctx:
+    """A libgift context: per-user keys on one device.  See include/gift.h for semantics."""
+
+    def __init__(self, max_users: int, device: int = 0, flags: int = 0):
+        import torch
+        if not torch.cuda.is_available():
+            raise RuntimeError("libgift needs a CUDA device; there is no CPU fallback")
+        self._h = C.c_void_p()
+        _check(lib().gift_ctx_create(C.byref(self._h), device, max_users, flags), "gift_ctx_create")
+        self.max_users = max_users
+        self.device = device
+
+    def close(self):
+        if self._h:
+            lib().gift_ctx_destroy(self._h)
+            self._h = C.c_void_p()
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+    def __enter__(self):
+        return self
+
+    def __exit__(self, *exc):
+        self.close()
+
+    def reserve(self, max_segs: int):
+        _check(lib().gift_ctx_reserve(self._h, max_segs), "gift_ctx_reserve")
+
+    def set_keys(self, user_ids, keys16, stream=None):
+        ids = np.ascontiguousarray(user_ids, dtype=np.int32)
+        keys = np.ascontiguousarray(keys16, dtype=np.uint8).reshape(-1)
+        if keys.size != 16 * ids.size:
+            raise ValueError("keys16 must hold 16 bytes per user id")
+        _check(lib().gift_set_keys(self._h, ids.ctypes.data_as(C.c_void_p), keys.ctypes.data_as(C.c_void_p),
+                                   ids.size, _stream_ptr(stream)), "gift_set_keys")
+
+    def clear_keys(self, user_ids, stream=None):
+        ids = np.ascontiguousarray(user_ids, dtype=np.int32)
+        _check(lib().gift_clear_keys(self._h, ids.ctypes.data_as(C.c_void_p), ids.size, _stream_ptr(stream)),
+               "gift_clear_keys")
+
+    @staticmethod
+    def _tables(page_table, page_bytes, owner_map, unit_bytes):
+        pg = lb = None
+        if page_table is not None:
+            pg = _Pages(page_table.data_ptr(), page_table.numel(), page_bytes)
+        if owner_map is not None:
+            lb = _Labels(owner_map.data_ptr(), owner_map.numel(), unit_bytes)
+        return pg, lb
+
+    def seg_encrypt(self, src, dst, segs, nseg, tags_out, status, page_table=None, page_bytes=0,
+                    owner_map=None, unit_bytes=0, stream=None):
+        pg, lb = self._tables(page_table, page_bytes, owner_map, unit_bytes)
+        _check(lib().gift_seg_encrypt(self._h, _dev(src), _dev(dst), src.numel() * src.element_size(), _dev(segs),
+                                      nseg, C.byref(pg) if pg else None, C.byref(lb) if lb else None,
+                                      _dev(tags_out), _dev(status), _stream_ptr(stream)), "gift_seg_encrypt")
+
+    def seg_decrypt(self, src, dst, segs, nseg, tags_in, status, page_table=None, page_bytes=0,
+                    owner_map=None, unit_bytes=0, stream=None):
+        pg, lb = self._tables(page_table, page_bytes, owner_map, unit_bytes)
+        _check(lib().gift_seg_decrypt(self._h, _dev(src), _dev(dst), src.numel() * src.element_size(), _dev(segs),
+                                      nseg, C.byref(pg) if pg else None, C.byref(lb) if lb else None,
+                                      _dev(tags_in), _dev(status), _stream_ptr(stream)), "gift_seg_decrypt")
+
+    def verify_tags(self, src, segs, nseg, tags_in, status, page_table=None, page_bytes=0, stream=None):
+        pg, _ = self._tables(page_table, page_bytes, None, 0)
+        _check(lib().gift_verify_tags(self._h, _dev(src), src.numel() * src.element_size(), _dev(segs), nseg,
+                                      C.byref(pg) if pg else None, _dev(tags_in), _dev(status),
+                                      _stream_ptr(stream)), "gift_verify_tags")
+
+    def propagate_labels(self, kind, in_maps, out_map, viol, *, n_out=None, param_mask=0, seg_ptr=None,
+                         src_ptr=None, src_idx=None, gather=None, stream=None):
+        n_out = out_map.numel() if n_out is None else n_out
+        n_seg = seg_ptr.numel() - 1 if seg_ptr is not None else 0
+        rule = _Rule(kind, n_out, len(in_maps), n_seg,
+                     in_maps[0].numel(), in_maps[1].numel() if len(in_maps) > 1 else 0,
+                     seg_ptr.data_ptr() if seg_ptr is not None else None,
+                     src_ptr.data_ptr() if src_ptr is not None else None,
+                     src_idx.data_ptr() if src_idx is not None else None,
+                     gather.data_ptr() if gather is not None else None, param_mask)
+        arr = (C.c_void_p * len(in_maps))(*[m.data_ptr() for m in in_maps])
+        _check(lib().gift_propagate_labels(self._h, C.byref(rule), arr, _dev(out_map), _dev(viol),
+                                           _stream_ptr(stream)), "gift_propagate_labels")
+
+    def launch_count(self) -> int:
+        return int(lib().gift_launch_count(self._h))
+
+    def timing_enable(self, on: bool = True):
+        _check(lib().gift_timing_enable(self._h, 1 if on else 0), "gift_timing_enable")
+
+    def timing_read(self):
+        """(total milliseconds, launches) of the cipher kernel since the last read."""
+        ms, n = C.c_double(), C.c_uint32()
+        _check(lib().gift_timing_read(self._h, C.byref(ms), C.byref(n)), "gift_timing_read")
+        return ms.value, n.value
+
+
+PROBE_KINDS = {0: "lop3", 1: "mad.wide.u32", 2: "prmt", 3: "ld.shared.u32", 4: "shf", 5: "add.u32",
+               6: "lop3+mad.wide", 7: "mad.lo.u32", 8: "lop3+ld.shared"}
+
+
+def probe_pipe(kind: int, iters: int = 2000, device: int = 0):
+    """(lane-operations per SM clock, SM MHz seen) for one instruction kind."""
+    ops, mhz = C.c_double(), C.c_double()
+    _check(lib().gift_probe_pipe(device, kind, iters, C.byref(ops), C.byref(mhz)), "gift_probe_pipe")
+    return ops.value, mhz.value

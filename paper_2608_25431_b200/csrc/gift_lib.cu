@@ -1,0 +1,1038 @@
+// libgift: context, kernels and C entry points (see include/gift.h).
+//
+// Call structure of gift_seg_encrypt / gift_seg_decrypt / gift_verify_tags, all
+// on the caller's stream with no host round trip in between:
+//   1. plan_kernel     one warp per segment: descriptor checks, ownership-label
+//                      check, pre-status, zeroed hash accumulators, block total
+//   2. scan_kernel     picks the run length from the block total and turns runs
+//                      per segment into a prefix sum (the work list)
+//   3. crypt_kernel    persistent warps pull runs from a counter; per run:
+//                      CTR keystream + XOR + GHASH; the warp that completes a
+//                      segment finishes its tag (no waiting, tickets only)
+//   4. fixup_kernel    decrypt only: zero-fills failed segments, marks their units
+//
+// AES uses T-tables replicated across the 32 shared-memory banks so that a warp's
+// 32 data-dependent lookups never conflict; GHASH uses masked integer multiplies
+// (gf128.cuh).  The path is bound by the integer pipes, not by HBM: at most about
+// one eighth of the memory bandwidth is needed, so data moves with plain 128-bit
+// loads and stores and no staging through shared memory.
+#include <cuda_runtime.h>
+#include <stdint.h>
+#include <stdio.h>
+#include <string.h>
+
+#include <new>
+
+#include "../../include/gift.h"
+#include "gift_core.cuh"
+
+using namespace gift;
+
+#define GIFT_VERSION 100u   // 0.1.0
+
+// ---------------------------------------------------------------------------
+// context
+// ---------------------------------------------------------------------------
+
+struct Globals {
+    unsigned long long total_blocks;   // 16-byte blocks of all accepted segments
+    uint32_t total_runs;
+    uint32_t run_blocks;               // blocks per run chosen for this call
+    uint32_t work;                     // next run to hand out
+    uint32_t pad[3];
+};
+
+struct gift_ctx {
+    int device;
+    uint32_t max_users;
+    uint32_t flags;
+    int chains;                        // Horner chains per lane (1 or 2)
+    int tables;                        // T-tables held in shared memory (2 or 4)
+    int num_sms;
+    uint32_t* d_t0;                    // 256-entry T0 in global memory
+    KeyHot* d_hot;                     // [max_users]
+    u128* d_pow;                       // [max_users][POW_LEVELS*256]
+    uint8_t* h_stage;                  // pinned staging for keys
+    uint32_t stage_cap;                // users the staging buffers hold
+    int32_t* d_stage_ids;
+    uint8_t* d_stage_keys;
+    uint32_t seg_cap;
+    uint32_t* d_run_prefix;            // [seg_cap + 1]
+    uint4* d_acc;                      // [seg_cap]
+    uint32_t* d_ticket;                // [seg_cap]
+    Globals* d_glob;
+    int32_t* d_snapshot;               // label snapshot for aliased rules
+    uint32_t snapshot_cap;
+    uint64_t launches;
+    int timing;                        // record events around the cipher kernel
+    uint32_t n_timed;
+    cudaEvent_t* ev;                   // 2 * MAX_TIMED events, created on first enable
+};
+
+#define MAX_TIMED 1024u
+
+#define CU_TRY(expr)                                   \
+    do {                                               \
+        cudaError_t e_ = (expr);                       \
+        if (e_ != cudaSuccess) {                       \
+            return e_ == cudaErrorMemoryAllocation ? GIFT_E_NOMEM : GIFT_E_CUDA; \
+        }                                              \
+    } while (0)
+
+namespace {
+
+// ---------------------------------------------------------------------------
+// tables and keys
+// ---------------------------------------------------------------------------
+
+__global__ void init_t0_kernel(uint32_t* t0)
+{
+    t0[threadIdx.x] = t0_entry(threadIdx.x);
+}
+
+// Four threads per user: each derives the key schedule and H, thread m builds
+// level m of the power table, thread 0 also stores the hot record.
+__global__ void key_setup_kernel(const uint32_t* __restrict__ t0, const int32_t* __restrict__ ids,
+                                 const uint8_t* __restrict__ keys, uint32_t n, KeyHot* hot, u128* pow)
+{
+    const uint32_t g = blockIdx.x * blockDim.x + threadIdx.x;
+    const uint32_t i = g / POW_LEVELS;
+    const int m = (int)(g % POW_LEVELS);
+    if (i >= n) return;
+    PlainTab tb;
+    tb.t0 = t0;
+    uint32_t key[4];
+    const Block kb = load_block(keys + 16 * (size_t)i);
+    key[0] = kb.d[0]; key[1] = kb.d[1]; key[2] = kb.d[2]; key[3] = kb.d[3];
+    KeyHot rec;
+    u128 h;
+    derive_key_hot(tb, key, &rec, &h);
+    const uint32_t u = (uint32_t)ids[i];
+    build_pow_level(h, m, pow + (size_t)u * (POW_LEVELS * 256) + m * 256);
+    if (m == 0) hot[u] = rec;
+}
+
+__global__ void key_clear_kernel(const int32_t* __restrict__ ids, uint32_t n, KeyHot* hot, u128* pow)
+{
+    const uint32_t i = blockIdx.x;
+    if (i >= n) return;
+    const uint32_t u = (uint32_t)ids[i];
+    uint32_t* h = reinterpret_cast<uint32_t*>(hot + u);
+    for (uint32_t k = threadIdx.x; k < sizeof(KeyHot) / 4; k += blockDim.x) h[k] = 0u;
+    uint32_t* p = reinterpret_cast<uint32_t*>(pow + (size_t)u * (POW_LEVELS * 256));
+    for (uint32_t k = threadIdx.x; k < POW_LEVELS * 256 * 4; k += blockDim.x) p[k] = 0u;
+}
+
+// ---------------------------------------------------------------------------
+// call parameters shared by the segment kernels
+// ---------------------------------------------------------------------------
+
+struct CallArgs {
+    const uint8_t* src;
+    uint8_t* dst;
+    uint64_t buf_bytes;
+    const gift_seg* segs;
+    uint32_t nseg;
+    const int32_t* page_table;     // nullptr: flat
+    uint32_t n_pages;
+    uint64_t page_bytes;
+    int32_t* owner_map;            // nullptr: no labels
+    uint32_t n_units;
+    uint64_t unit_bytes;
+    uint8_t* tags;                 // out (encrypt) or in (decrypt, verify)
+    uint32_t* status;
+    const KeyHot* hot;
+    const u128* pow;
+    uint32_t max_users;
+    uint32_t* run_prefix;
+    uint4* acc;
+    uint32_t* ticket;
+    Globals* glob;
+    uint32_t target_runs;          // runs wanted for a balanced call
+    uint32_t max_run_blocks;
+    uint32_t min_run_blocks;
+};
+
+__device__ __forceinline__ uint64_t seg_blocks(uint64_t len) { return (len + 15) >> 4; }
+
+// Units a segment covers: flat, [u0, u0 + count); paged, one per page.
+__device__ __forceinline__ uint64_t seg_unit_count(const CallArgs& a, const gift_seg& s, uint64_t* u0)
+{
+    if (s.len == 0) { *u0 = 0; return 0; }
+    if (a.page_table == nullptr) {
+        *u0 = s.offset / a.unit_bytes;
+        const uint64_t u1 = (s.offset + s.len + a.unit_bytes - 1) / a.unit_bytes;
+        return u1 - *u0;
+    }
+    *u0 = 0;
+    return (s.len + a.page_bytes - 1) / a.page_bytes;
+}
+
+__device__ __forceinline__ uint64_t seg_unit(const CallArgs& a, const gift_seg& s, uint64_t u0, uint64_t k)
+{
+    if (a.page_table == nullptr) return u0 + k;
+    return (uint64_t)(uint32_t)a.page_table[(uint64_t)s.page0 + k];
+}
+
+// ---------------------------------------------------------------------------
+// 1. plan: validation, label check (paper sec. 3 step 4, sec. 4.2), pre-status
+// ---------------------------------------------------------------------------
+
+template <int MODE>
+__global__ void plan_kernel(CallArgs a)
+{
+    const int lane = threadIdx.x & 31;
+    const uint32_t s = (blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+    if (s >= a.nseg) return;
+    const gift_seg seg = a.segs[s];
+    const bool labels = a.owner_map != nullptr;
+
+    bool bad = seg.flags != 0 || seg.len > GIFT_MAX_SEG_BYTES;
+    if (!bad) {
+        if (a.page_table == nullptr) {
+            bad = (seg.offset & 15) != 0 || seg.offset > a.buf_bytes || seg.len > a.buf_bytes - seg.offset;
+            if (!bad && labels && seg.len > 0) {
+                const uint64_t u1 = (seg.offset + seg.len + a.unit_bytes - 1) / a.unit_bytes;
+                bad = u1 > a.n_units;
+            }
+        } else {
+            const uint64_t np = (seg.len + a.page_bytes - 1) / a.page_bytes;
+            bad = (uint64_t)seg.page0 + np > a.n_pages;
+            if (!bad) {
+                bool b = false;
+                for (uint64_t k = lane; k < np; k += 32) {
+                    const int32_t t = a.page_table[(uint64_t)seg.page0 + k];
+                    b |= t < 0 || ((uint64_t)t + 1) * a.page_bytes > a.buf_bytes ||
+                         (labels && (uint64_t)t >= a.n_units);
+                }
+                bad = __any_sync(0xFFFFFFFFu, b);
+            }
+        }
+    }
+    uint32_t st = 0;
+    if (bad) {
+        st = GIFT_ST_BAD_DESC;
+    } else {
+        if (MODE == MODE_ENCRYPT && labels) {
+            uint64_t u0;
+            const uint64_t nu = seg_unit_count(a, seg, &u0);
+            bool unowned = false, mism = false;
+            for (uint64_t k = lane; k < nu; k += 32) {
+                const int32_t l = a.owner_map[seg_unit(a, seg, u0, k)];
+                unowned |= l <= GIFT_OWNER_NONE;
+                mism |= l == GIFT_OWNER_PARAM || (l >= 0 && l != seg.owner);
+            }
+            if (__any_sync(0xFFFFFFFFu, unowned)) st |= GIFT_ST_UNOWNED;
+            if (__any_sync(0xFFFFFFFFu, mism)) st |= GIFT_ST_OWNER_MISMATCH;
+        }
+        const bool has_key = seg.owner >= 0 && (uint32_t)seg.owner < a.max_users && a.hot[seg.owner].valid != 0;
+        if (!has_key) st |= GIFT_ST_NO_KEY;
+    }
+    if (lane == 0) {
+        a.status[s] = st;
+        a.acc[s] = make_uint4(0u, 0u, 0u, 0u);
+        a.ticket[s] = 0u;
+        if (st == 0) {
+            const uint64_t nb = seg_blocks(seg.len);
+            atomicAdd(&a.glob->total_blocks, (unsigned long long)(nb ? nb : 1));
+        } else if (MODE == MODE_ENCRYPT) {
+            reinterpret_cast<uint4*>(a.tags)[s] = make_uint4(0u, 0u, 0u, 0u);
+        }
+    }
+}
+
+// ---------------------------------------------------------------------------
+// 2. scan: run length and work list
+// ---------------------------------------------------------------------------
+
+__device__ __forceinline__ uint32_t runs_of(uint64_t len, uint32_t st, uint32_t run_blocks)
+{
+    if (st != 0) return 0u;
+    const uint64_t nb = seg_blocks(len);
+    const uint64_t r = (nb + run_blocks - 1) / run_blocks;
+    return r ? (uint32_t)r : 1u;      // an empty segment still needs its tag finished
+}
+
+__global__ void scan_kernel(CallArgs a)
+{
+    __shared__ uint32_t warp_sums[32];
+    __shared__ uint32_t carry;
+    __shared__ uint32_t run_blocks_s;
+    const int tid = threadIdx.x, lane = tid & 31, wid = tid >> 5;
+    if (tid == 0) {
+        // smallest power of two that keeps the run count near the target, within limits
+        const unsigned long long total = a.glob->total_blocks;
+        uint32_t rb = a.min_run_blocks;
+        while (rb < a.max_run_blocks && total / rb > a.target_runs) rb <<= 1;
+        run_blocks_s = rb;
+        carry = 0u;
+    }
+    __syncthreads();
+    const uint32_t rb = run_blocks_s;
+    for (uint32_t base = 0; base < a.nseg; base += blockDim.x) {
+        const uint32_t i = base + tid;
+        uint32_t v = 0;
+        if (i < a.nseg) v = runs_of(a.segs[i].len, a.status[i], rb);
+        uint32_t x = v;
+        for (int o = 1; o < 32; o <<= 1) {
+            const uint32_t y = __shfl_up_sync(0xFFFFFFFFu, x, o);
+            if (lane >= o) x += y;
+        }
+        if (lane == 31) warp_sums[wid] = x;
+        __syncthreads();
+        if (wid == 0) {
+            uint32_t w = lane < (int)(blockDim.x >> 5) ? warp_sums[lane] : 0u;
+            for (int o = 1; o < 32; o <<= 1) {
+                const uint32_t y = __shfl_up_sync(0xFFFFFFFFu, w, o);
+                if (lane >= o) w += y;
+            }
+            warp_sums[lane] = w;      // inclusive sums of the warps
+        }
+        __syncthreads();
+        const uint32_t before = carry + (wid ? warp_sums[wid - 1] : 0u) + (x - v);
+        if (i < a.nseg) a.run_prefix[i] = before;
+        __syncthreads();
+        if (tid == 0) carry += warp_sums[(blockDim.x >> 5) - 1];
+        __syncthreads();
+    }
+    if (tid == 0) {
+        a.run_prefix[a.nseg] = carry;
+        a.glob->total_runs = carry;
+        a.glob->run_blocks = rb;
+        a.glob->work = 0u;
+    }
+}
+
+// ---------------------------------------------------------------------------
+// 3. crypt: the hot loop
+// ---------------------------------------------------------------------------
+
+extern __shared__ __align__(16) unsigned char smem_raw[];
+
+// T-tables in shared memory, one copy per bank.  Entry x of table t for lane l is
+// the word at byte  (t>>1)*65536 + x*256 + (t&1)*128 + l*4 : the index lands in
+// byte 1 of the offset, so one byte-permute builds the address and the bank is
+// always the lane's own.  With NT == 2 only T0 and T1 are stored; T2 and T3 are
+// their 16-bit rotations.
+template <int NT>
+struct SmemTab {
+    uint32_t lb0, lb1;     // lane*4 and lane*4 + 128
+    template <int T, int K>
+    __device__ __forceinline__ uint32_t look(uint32_t w) const
+    {
+        if (NT == 4) {
+            const uint32_t off = __byte_perm(w, (T & 1) ? lb1 : lb0, 0x7604u | (K << 4));
+            return *reinterpret_cast<const uint32_t*>(smem_raw + (T >> 1) * 65536 + off);
+        } else {
+            const uint32_t off = __byte_perm(w, (T & 1) ? lb1 : lb0, 0x7604u | (K << 4));
+            const uint32_t v = *reinterpret_cast<const uint32_t*>(smem_raw + off);
+            return (T >> 1) ? __byte_perm(v, 0u, 0x1032u) : v;
+        }
+    }
+    template <int K>
+    __device__ __forceinline__ uint32_t sub(uint32_t w) const
+    {
+        const uint32_t off = __byte_perm(w, lb0, 0x7604u | (K << 4));
+        return *reinterpret_cast<const uint32_t*>(smem_raw + off);
+    }
+};
+
+template <int NT>
+__device__ __forceinline__ void fill_tables(const uint32_t* __restrict__ t0)
+{
+    // word index inside a 64 KiB chunk: x*64 + parity*32 + lane
+    uint32_t* tabs = reinterpret_cast<uint32_t*>(smem_raw);
+    constexpr int chunks = NT == 4 ? 2 : 1;
+    for (uint32_t idx = threadIdx.x; idx < chunks * 16384u; idx += blockDim.x) {
+        const uint32_t chunk = idx >> 14, x = (idx >> 6) & 255u, parity = (idx >> 5) & 1u;
+        const uint32_t t = chunk * 2 + parity;
+        tabs[idx] = rotl32(t0[x], 8 * (int)t);
+    }
+}
+
+__device__ __forceinline__ uint32_t warp_xor(uint32_t v)
+{
+    for (int o = 16; o > 0; o >>= 1) v ^= __shfl_xor_sync(0xFFFFFFFFu, v, o);
+    return v;
+}
+
+template <int U, int MODE, int NT>
+__global__ void __launch_bounds__(512, 1) crypt_kernel(CallArgs a, const uint32_t* __restrict__ t0)
+{
+    constexpr uint32_t TAB_BYTES = NT == 4 ? 131072u : 65536u;
+    const int lane = threadIdx.x & 31, wid = threadIdx.x >> 5;
+    fill_tables<NT>(t0);
+    __syncthreads();
+    SmemTab<NT> tb;
+    tb.lb0 = (uint32_t)lane * 4u;
+    tb.lb1 = (uint32_t)lane * 4u + 128u;
+    KeyHot* slot = reinterpret_cast<KeyHot*>(smem_raw + TAB_BYTES) + wid;
+
+    const uint32_t total_runs = a.glob->total_runs;
+    const uint32_t run_blocks = a.glob->run_blocks;
+    for (;;) {
+        uint32_t run = 0;
+        if (lane == 0) run = atomicAdd(&a.glob->work, 1u);
+        run = __shfl_sync(0xFFFFFFFFu, run, 0);
+        if (run >= total_runs) break;
+        // segment of this run: the largest s with run_prefix[s] <= run
+        uint32_t lo = 0, hi = a.nseg;
+        while (hi - lo > 1) {
+            const uint32_t mid = (lo + hi) >> 1;
+            if (a.run_prefix[mid] <= run) lo = mid; else hi = mid;
+        }
+        const uint32_t s = lo;
+        const uint32_t first_run = a.run_prefix[s];
+        const uint32_t seg_runs = a.run_prefix[s + 1] - first_run;
+        const gift_seg seg = a.segs[s];
+        const uint64_t nblk = seg_blocks(seg.len);
+        const uint64_t run_first = (uint64_t)(run - first_run) * run_blocks;
+        const uint64_t left = nblk - run_first;
+        const uint32_t run_n = left < run_blocks ? (uint32_t)left : run_blocks;
+
+        // this warp's copy of the owner's key material (512 bytes: one uint4 per lane)
+        __syncwarp();
+        reinterpret_cast<uint4*>(slot)[lane] = reinterpret_cast<const uint4*>(a.hot + seg.owner)[lane];
+        __syncwarp();
+        const uint32_t* rk = slot->rk;
+        uint32_t nonce[3];
+        nonce[0] = (uint32_t)seg.nonce[0] | ((uint32_t)seg.nonce[1] << 8) | ((uint32_t)seg.nonce[2] << 16) | ((uint32_t)seg.nonce[3] << 24);
+        nonce[1] = (uint32_t)seg.nonce[4] | ((uint32_t)seg.nonce[5] << 8) | ((uint32_t)seg.nonce[6] << 16) | ((uint32_t)seg.nonce[7] << 24);
+        nonce[2] = (uint32_t)seg.nonce[8] | ((uint32_t)seg.nonce[9] << 8) | ((uint32_t)seg.nonce[10] << 16) | ((uint32_t)seg.nonce[11] << 24);
+        const CtrPrefix pre = ctr_prefix(tb, rk, nonce);
+        SegAddr addr;
+        addr.table = a.page_table;
+        addr.page_bytes = a.page_bytes;
+        addr.origin = a.page_table ? (uint64_t)seg.page0 : seg.offset;
+
+        const u128 part = run_lane<U, MODE>(tb, rk, pre, slot->hs[U - 1],
+                                            a.pow + (size_t)seg.owner * (POW_LEVELS * 256), a.src, a.dst, addr,
+                                            nblk, run_first, run_n, (uint32_t)(seg.len & 15), lane);
+        u128 sum;
+        sum.w[0] = warp_xor(part.w[0]);
+        sum.w[1] = warp_xor(part.w[1]);
+        sum.w[2] = warp_xor(part.w[2]);
+        sum.w[3] = warp_xor(part.w[3]);
+
+        // combine the runs of a segment: XOR is order-free, the last arrival finishes
+        bool last = true;
+        if (seg_runs > 1) {
+            uint32_t t = 0;
+            if (lane == 0) {
+                uint32_t* acc = reinterpret_cast<uint32_t*>(a.acc + s);
+                atomicXor(acc + 0, sum.w[0]);
+                atomicXor(acc + 1, sum.w[1]);
+                atomicXor(acc + 2, sum.w[2]);
+                atomicXor(acc + 3, sum.w[3]);
+                __threadfence();
+                t = atomicAdd(a.ticket + s, 1u);
+            }
+            t = __shfl_sync(0xFFFFFFFFu, t, 0);
+            last = t == seg_runs - 1;
+            if (last) {
+                __threadfence();
+                uint32_t* acc = reinterpret_cast<uint32_t*>(a.acc + s);
+                if (lane < 4) sum.w[0] = atomicOr(acc + lane, 0u);
+                const uint32_t v = sum.w[0];
+                sum.w[0] = __shfl_sync(0xFFFFFFFFu, v, 0);
+                sum.w[1] = __shfl_sync(0xFFFFFFFFu, v, 1);
+                sum.w[2] = __shfl_sync(0xFFFFFFFFu, v, 2);
+                sum.w[3] = __shfl_sync(0xFFFFFFFFu, v, 3);
+            }
+        }
+        if (last) {
+            uint32_t tag[4];
+            finish_tag(tb, rk, slot->h, nonce, seg.len, sum, tag);
+            uint4* tagp = reinterpret_cast<uint4*>(a.tags) + s;
+            if (MODE == MODE_ENCRYPT) {
+                if (lane == 0) *tagp = make_uint4(tag[0], tag[1], tag[2], tag[3]);
+            } else {
+                const uint4 given = *tagp;
+                const bool ok = given.x == tag[0] && given.y == tag[1] && given.z == tag[2] && given.w == tag[3];
+                if (lane == 0 && !ok) a.status[s] = GIFT_ST_TAG_MISMATCH;
+                if (MODE == MODE_DECRYPT && ok && a.owner_map != nullptr) {
+                    // import succeeded: record the claimed owner on the covered units
+                    uint64_t u0;
+                    const uint64_t nu = seg_unit_count(a, seg, &u0);
+                    for (uint64_t k = lane; k < nu; k += 32) a.owner_map[seg_unit(a, seg, u0, k)] = seg.owner;
+                }
+            }
+        }
+    }
+}
+
+// ---------------------------------------------------------------------------
+// 4. fix-up after decrypt: failed segments read as zeros and become unowned
+// ---------------------------------------------------------------------------
+
+__global__ void fixup_kernel(CallArgs a)
+{
+    for (uint32_t s = blockIdx.x; s < a.nseg; s += gridDim.x) {
+        const uint32_t st = a.status[s];
+        if ((st & (GIFT_ST_TAG_MISMATCH | GIFT_ST_NO_KEY)) == 0 || (st & GIFT_ST_BAD_DESC)) continue;
+        const gift_seg seg = a.segs[s];
+        const uint64_t full = seg.len >> 4;
+        if (a.page_table == nullptr) {
+            uint4* p = reinterpret_cast<uint4*>(a.dst + seg.offset);
+            for (uint64_t k = threadIdx.x; k < full; k += blockDim.x) p[k] = make_uint4(0u, 0u, 0u, 0u);
+            for (uint64_t k = (full << 4) + threadIdx.x; k < seg.len; k += blockDim.x) a.dst[seg.offset + k] = 0;
+        } else {
+            const uint64_t per_page = a.page_bytes >> 4;
+            for (uint64_t k = threadIdx.x; k < full; k += blockDim.x) {
+                const uint64_t pg = k / per_page, in = k - pg * per_page;
+                const uint64_t base = (uint64_t)(uint32_t)a.page_table[(uint64_t)seg.page0 + pg] * a.page_bytes;
+                reinterpret_cast<uint4*>(a.dst + base)[in] = make_uint4(0u, 0u, 0u, 0u);
+            }
+            for (uint64_t k = (full << 4) + threadIdx.x; k < seg.len; k += blockDim.x) {
+                const uint64_t pg = k / a.page_bytes, in = k - pg * a.page_bytes;
+                const uint64_t base = (uint64_t)(uint32_t)a.page_table[(uint64_t)seg.page0 + pg] * a.page_bytes;
+                a.dst[base + in] = 0;
+            }
+        }
+        if (a.owner_map != nullptr) {
+            uint64_t u0;
+            const uint64_t nu = seg_unit_count(a, seg, &u0);
+            for (uint64_t k = threadIdx.x; k < nu; k += blockDim.x)
+                a.owner_map[seg_unit(a, seg, u0, k)] = GIFT_OWNER_NONE;
+        }
+    }
+}
+
+// ---------------------------------------------------------------------------
+// label propagation (paper sec. 4.3, rule steps 4 and 5)
+// ---------------------------------------------------------------------------
+
+struct RuleArgs {
+    uint32_t kind, n_out, n_in, n_seg, n_in0, n_in1, param_mask;
+    const int32_t* in[8];
+    const int32_t* seg_ptr;
+    const int32_t* src_ptr;
+    const int32_t* src_idx;
+    const int32_t* gather;
+    int32_t* out;
+    uint32_t* viol;
+};
+
+// The join over a set of labels is decided by three facts: was any label NONE or
+// CONFLICT, the smallest user id seen and the largest one (PARAM is neutral).
+struct JoinAcc {
+    bool bad;
+    int32_t lo, hi;
+    __device__ __forceinline__ void init() { bad = false; lo = 0x7FFFFFFF; hi = -1; }
+    __device__ __forceinline__ void add(int32_t l)
+    {
+        if (l <= GIFT_OWNER_NONE) bad = true;
+        else if (l >= 0) { lo = min(lo, l); hi = max(hi, l); }
+    }
+    __device__ __forceinline__ int32_t result() const
+    {
+        if (bad) return GIFT_OWNER_CONFLICT;
+        if (hi < 0) return GIFT_OWNER_PARAM;
+        return lo == hi ? lo : GIFT_OWNER_CONFLICT;
+    }
+};
+
+__device__ __forceinline__ void report_violation(uint32_t* viol, bool conflict, uint32_t j)
+{
+    const uint32_t m = __ballot_sync(__activemask(), conflict);
+    if (conflict) {
+        const int leader = __ffs(m) - 1;
+        if ((int)(threadIdx.x & 31) == leader) {
+            atomicAdd(viol, (uint32_t)__popc(m));
+            atomicMin(viol + 1, j);      // the leader holds the smallest index of its warp
+        }
+    }
+}
+
+__global__ void rule_pointwise_kernel(RuleArgs r)
+{
+    const uint32_t j = blockIdx.x * blockDim.x + threadIdx.x;
+    if (j >= r.n_out) return;
+    JoinAcc acc;
+    acc.init();
+    if (r.kind == GIFT_RULE_IDENTITY) {
+        acc.add(r.in[0][j]);
+    } else if (r.kind == GIFT_RULE_BROADCAST) {
+        const int32_t g = r.gather[j];
+        if (g < 0 || (uint32_t)g >= r.n_in0) acc.bad = true; else acc.add(r.in[0][g]);
+    } else {   // ROWWISE
+        for (uint32_t k = 0; k < r.n_in; k++) {
+            if ((r.param_mask >> k) & 1u) {
+                if (r.in[k][0] != GIFT_OWNER_PARAM) acc.bad = true;   // step 4: parameter operand mislabelled
+            } else {
+                acc.add(r.in[k][j]);
+            }
+        }
+    }
+    const int32_t o = acc.result();
+    r.out[j] = o;
+    report_violation(r.viol, o == GIFT_OWNER_CONFLICT, j);
+}
+
+// One warp per reduction segment; outputs outside every segment become CONFLICT.
+__global__ void rule_segreduce_kernel(RuleArgs r)
+{
+    const int lane = threadIdx.x & 31;
+    const uint32_t w = (blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+    if (w < r.n_seg) {
+        const int32_t t0 = r.seg_ptr[w], t1 = r.seg_ptr[w + 1];
+        const int32_t e0 = r.src_ptr[w], e1 = r.src_ptr[w + 1];
+        JoinAcc acc;
+        acc.init();
+        for (int32_t t = t0 + lane; t < t1; t += 32) acc.add(r.in[0][t]);
+        for (int32_t e = e0 + lane; e < e1; e += 32) {
+            const int32_t b = r.src_idx[e];
+            if (b < 0 || (uint32_t)b >= r.n_in1) acc.bad = true; else acc.add(r.in[1][b]);
+        }
+        acc.bad = __any_sync(0xFFFFFFFFu, acc.bad);
+        acc.lo = __reduce_min_sync(0xFFFFFFFFu, acc.lo);
+        acc.hi = __reduce_max_sync(0xFFFFFFFFu, acc.hi);
+        const int32_t m = acc.result();
+        __syncwarp();
+        for (int32_t t = t0 + lane; t < t1; t += 32) r.out[t] = m;
+        if (m == GIFT_OWNER_CONFLICT && lane == 0 && t1 > t0) {
+            atomicAdd(r.viol, (uint32_t)(t1 - t0));
+            atomicMin(r.viol + 1, (uint32_t)t0);
+        }
+    } else {
+        // threads past the segments cover the outputs before the first and after the last segment
+        const uint32_t extra = (blockIdx.x * blockDim.x + threadIdx.x) - r.n_seg * 32u;
+        const uint32_t head = (uint32_t)r.seg_ptr[0];
+        const uint32_t tail0 = (uint32_t)r.seg_ptr[r.n_seg];
+        const uint32_t n_extra = head + (r.n_out - tail0);
+        if (extra < n_extra) {
+            const uint32_t j = extra < head ? extra : tail0 + (extra - head);
+            r.out[j] = GIFT_OWNER_CONFLICT;
+            atomicAdd(r.viol, 1u);
+            atomicMin(r.viol + 1, j);
+        }
+    }
+}
+
+__global__ void viol_init_kernel(uint32_t* viol)
+{
+    viol[0] = 0u;
+    viol[1] = 0xFFFFFFFFu;
+}
+
+// ---------------------------------------------------------------------------
+// host side
+// ---------------------------------------------------------------------------
+
+struct DeviceGuard {
+    int prev;
+    bool ok;
+    explicit DeviceGuard(int dev) : prev(-1), ok(false)
+    {
+        if (cudaGetDevice(&prev) != cudaSuccess) return;
+        ok = prev == dev || cudaSetDevice(dev) == cudaSuccess;
+    }
+    ~DeviceGuard()
+    {
+        if (ok && prev >= 0) cudaSetDevice(prev);
+    }
+};
+
+int ensure_scratch(gift_ctx* c, uint32_t nseg)
+{
+    if (nseg <= c->seg_cap) return GIFT_OK;
+    uint32_t cap = c->seg_cap ? c->seg_cap : 1024u;
+    while (cap < nseg) cap = cap > 0x7FFFFFFFu ? nseg : cap * 2u;
+    CU_TRY(cudaDeviceSynchronize());
+    cudaFree(c->d_run_prefix);
+    cudaFree(c->d_acc);
+    cudaFree(c->d_ticket);
+    c->d_run_prefix = nullptr; c->d_acc = nullptr; c->d_ticket = nullptr;
+    c->seg_cap = 0;
+    CU_TRY(cudaMalloc(&c->d_run_prefix, ((size_t)cap + 1) * sizeof(uint32_t)));
+    CU_TRY(cudaMalloc(&c->d_acc, (size_t)cap * sizeof(uint4)));
+    CU_TRY(cudaMalloc(&c->d_ticket, (size_t)cap * sizeof(uint32_t)));
+    c->seg_cap = cap;
+    return GIFT_OK;
+}
+
+size_t crypt_smem_bytes(int tables)
+{
+    return (tables == 4 ? 131072u : 65536u) + 16u * sizeof(KeyHot);
+}
+
+template <int U, int MODE, int NT>
+int launch_crypt_t(gift_ctx* c, const CallArgs& a, cudaStream_t st)
+{
+    const size_t smem = crypt_smem_bytes(NT);
+    static bool configured[8] = {false, false, false, false, false, false, false, false};
+    auto kern = crypt_kernel<U, MODE, NT>;
+    if (c->device < 8 && !configured[c->device]) {
+        CU_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+        configured[c->device] = true;
+    } else if (c->device >= 8) {
+        CU_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+    }
+    const bool timed = c->timing && c->ev && c->n_timed < MAX_TIMED;
+    if (timed) CU_TRY(cudaEventRecord(c->ev[2 * c->n_timed], st));
+    kern<<<c->num_sms, 512, smem, st>>>(a, c->d_t0);
+    if (timed) {
+        CU_TRY(cudaEventRecord(c->ev[2 * c->n_timed + 1], st));
+        c->n_timed++;
+    }
+    c->launches++;
+    return GIFT_OK;
+}
+
+template <int MODE>
+int launch_crypt(gift_ctx* c, const CallArgs& a, cudaStream_t st)
+{
+    if (c->tables == 4) {
+        return c->chains == 2 ? launch_crypt_t<2, MODE, 4>(c, a, st) : launch_crypt_t<1, MODE, 4>(c, a, st);
+    }
+    return c->chains == 2 ? launch_crypt_t<2, MODE, 2>(c, a, st) : launch_crypt_t<1, MODE, 2>(c, a, st);
+}
+
+template <int MODE>
+int seg_call(gift_ctx* c, const void* src, void* dst, uint64_t buf_bytes, const gift_seg* segs, uint32_t nseg,
+             const gift_pages* pages, const gift_labels* labels, uint8_t* tags, uint32_t* status, void* stream)
+{
+    if (!c || !segs || !tags || !status) return nseg == 0 && c ? GIFT_OK : GIFT_E_INVAL;
+    if (nseg == 0) return GIFT_OK;
+    if (!src || (MODE != MODE_VERIFY && !dst)) return GIFT_E_INVAL;
+    if (((uintptr_t)src & 15) || ((uintptr_t)dst & 15) || ((uintptr_t)tags & 15)) return GIFT_E_ALIGN;
+    if (pages && (!pages->table || pages->page_bytes == 0)) return GIFT_E_INVAL;
+    if (pages && (pages->page_bytes & 15)) return GIFT_E_ALIGN;
+    if (labels && (!labels->owner_map || (!pages && labels->unit_bytes == 0))) return GIFT_E_INVAL;
+    DeviceGuard g(c->device);
+    if (!g.ok) return GIFT_E_CUDA;
+    int rc = ensure_scratch(c, nseg);
+    if (rc != GIFT_OK) return rc;
+    cudaStream_t st = (cudaStream_t)stream;
+
+    CallArgs a;
+    memset(&a, 0, sizeof(a));
+    a.src = (const uint8_t*)src;
+    a.dst = (uint8_t*)dst;
+    a.buf_bytes = buf_bytes;
+    a.segs = segs;
+    a.nseg = nseg;
+    if (pages) { a.page_table = pages->table; a.n_pages = pages->n; a.page_bytes = pages->page_bytes; }
+    if (labels) { a.owner_map = labels->owner_map; a.n_units = labels->n_units; a.unit_bytes = labels->unit_bytes; }
+    a.tags = tags;
+    a.status = status;
+    a.hot = c->d_hot;
+    a.pow = c->d_pow;
+    a.max_users = c->max_users;
+    a.run_prefix = c->d_run_prefix;
+    a.acc = c->d_acc;
+    a.ticket = c->d_ticket;
+    a.glob = c->d_glob;
+    a.target_runs = (uint32_t)c->num_sms * 16u * 8u;     // about eight runs per resident warp
+    a.max_run_blocks = 4096u;                             // 64 KiB
+    a.min_run_blocks = 256u;                              // 4 KiB
+
+    CU_TRY(cudaMemsetAsync(c->d_glob, 0, sizeof(Globals), st));
+    const uint32_t plan_blocks = (nseg + 7) / 8;          // 8 warps per block, one warp per segment
+    plan_kernel<MODE><<<plan_blocks, 256, 0, st>>>(a);
+    scan_kernel<<<1, 1024, 0, st>>>(a);
+    c->launches += 2;
+    rc = launch_crypt<MODE>(c, a, st);
+    if (rc != GIFT_OK) return rc;
+    if (MODE == MODE_DECRYPT) {
+        uint32_t fb = nseg < (uint32_t)c->num_sms * 8u ? nseg : (uint32_t)c->num_sms * 8u;
+        fixup_kernel<<<fb, 256, 0, st>>>(a);
+        c->launches++;
+    }
+    CU_TRY(cudaGetLastError());
+    return GIFT_OK;
+}
+
+bool ranges_overlap(const void* a, size_t na, const void* b, size_t nb)
+{
+    const uintptr_t a0 = (uintptr_t)a, b0 = (uintptr_t)b;
+    return a0 < b0 + nb && b0 < a0 + na;
+}
+
+}  // namespace
+
+// ---------------------------------------------------------------------------
+// C entry points
+// ---------------------------------------------------------------------------
+
+extern "C" {
+
+int gift_ctx_create(gift_ctx** out, int device, uint32_t max_users, uint32_t flags)
+{
+    if (!out || max_users == 0) return GIFT_E_INVAL;
+    *out = nullptr;
+    int chains = (int)(flags & 0xFu), tables = (int)((flags >> 4) & 0xFu);
+    if (chains == 0) chains = 2;
+    if (tables == 0) tables = 4;
+    if ((chains != 1 && chains != 2) || (tables != 2 && tables != 4) || (flags >> 8)) return GIFT_E_INVAL;
+    if (max_users > (1u << 20)) return GIFT_E_RANGE;
+    DeviceGuard g(device);
+    if (!g.ok) return GIFT_E_CUDA;
+    gift_ctx* c = new (std::nothrow) gift_ctx();
+    if (!c) return GIFT_E_NOMEM;
+    memset(c, 0, sizeof(*c));
+    c->device = device;
+    c->max_users = max_users;
+    c->flags = flags;
+    c->chains = chains;
+    c->tables = tables;
+    int rc = GIFT_OK;
+    cudaDeviceProp prop;
+    if (cudaGetDeviceProperties(&prop, device) != cudaSuccess) { delete c; return GIFT_E_CUDA; }
+    c->num_sms = prop.multiProcessorCount;
+    auto fail = [&](int code) { gift_ctx_destroy(c); return code; };
+    if (cudaMalloc(&c->d_t0, 256 * sizeof(uint32_t)) != cudaSuccess) return fail(GIFT_E_NOMEM);
+    if (cudaMalloc(&c->d_hot, (size_t)max_users * sizeof(KeyHot)) != cudaSuccess) return fail(GIFT_E_NOMEM);
+    if (cudaMalloc(&c->d_pow, (size_t)max_users * POW_LEVELS * 256 * sizeof(u128)) != cudaSuccess) return fail(GIFT_E_NOMEM);
+    if (cudaMalloc(&c->d_glob, sizeof(Globals)) != cudaSuccess) return fail(GIFT_E_NOMEM);
+    if (cudaMemset(c->d_hot, 0, (size_t)max_users * sizeof(KeyHot)) != cudaSuccess) return fail(GIFT_E_CUDA);
+    if (cudaMemset(c->d_pow, 0, (size_t)max_users * POW_LEVELS * 256 * sizeof(u128)) != cudaSuccess) return fail(GIFT_E_CUDA);
+    if (cudaMemset(c->d_glob, 0, sizeof(Globals)) != cudaSuccess) return fail(GIFT_E_CUDA);
+    init_t0_kernel<<<1, 256>>>(c->d_t0);
+    c->launches++;
+    if (cudaDeviceSynchronize() != cudaSuccess) return fail(GIFT_E_CUDA);
+    rc = ensure_scratch(c, 1024);
+    if (rc != GIFT_OK) return fail(rc);
+    *out = c;
+    return GIFT_OK;
+}
+
+int gift_ctx_destroy(gift_ctx* c)
+{
+    if (!c) return GIFT_E_INVAL;
+    DeviceGuard g(c->device);
+    if (g.ok) {
+        cudaDeviceSynchronize();
+        if (c->d_hot) cudaMemset(c->d_hot, 0, (size_t)c->max_users * sizeof(KeyHot));
+        if (c->d_pow) cudaMemset(c->d_pow, 0, (size_t)c->max_users * POW_LEVELS * 256 * sizeof(u128));
+        if (c->d_stage_keys) cudaMemset(c->d_stage_keys, 0, (size_t)c->stage_cap * 16);
+        cudaDeviceSynchronize();
+        cudaFree(c->d_t0); cudaFree(c->d_hot); cudaFree(c->d_pow); cudaFree(c->d_glob);
+        cudaFree(c->d_run_prefix); cudaFree(c->d_acc); cudaFree(c->d_ticket);
+        cudaFree(c->d_stage_ids); cudaFree(c->d_stage_keys); cudaFree(c->d_snapshot);
+        if (c->h_stage) {
+            memset(c->h_stage, 0, (size_t)c->stage_cap * 20);
+            cudaFreeHost(c->h_stage);
+        }
+        if (c->ev) {
+            for (uint32_t i = 0; i < 2 * MAX_TIMED; i++) cudaEventDestroy(c->ev[i]);
+            delete[] c->ev;
+        }
+    }
+    delete c;
+    return GIFT_OK;
+}
+
+int gift_ctx_reserve(gift_ctx* c, uint32_t max_segs)
+{
+    if (!c) return GIFT_E_INVAL;
+    DeviceGuard g(c->device);
+    if (!g.ok) return GIFT_E_CUDA;
+    return ensure_scratch(c, max_segs);
+}
+
+static int stage_ids(gift_ctx* c, const int32_t* user_ids, const uint8_t* keys16, uint32_t n, cudaStream_t st)
+{
+    for (uint32_t i = 0; i < n; i++)
+        if (user_ids[i] < 0 || (uint32_t)user_ids[i] >= c->max_users) return GIFT_E_RANGE;
+    if (n > c->stage_cap) {
+        CU_TRY(cudaDeviceSynchronize());
+        if (c->h_stage) { memset(c->h_stage, 0, (size_t)c->stage_cap * 20); cudaFreeHost(c->h_stage); c->h_stage = nullptr; }
+        cudaFree(c->d_stage_ids); cudaFree(c->d_stage_keys);
+        c->d_stage_ids = nullptr; c->d_stage_keys = nullptr; c->stage_cap = 0;
+        CU_TRY(cudaMallocHost(&c->h_stage, (size_t)n * 20));
+        CU_TRY(cudaMalloc(&c->d_stage_ids, (size_t)n * 4));
+        CU_TRY(cudaMalloc(&c->d_stage_keys, (size_t)n * 16));
+        c->stage_cap = n;
+    } else {
+        // the staging buffers may still be in use by an earlier call on another stream
+        CU_TRY(cudaDeviceSynchronize());
+    }
+    memcpy(c->h_stage, user_ids, (size_t)n * 4);
+    CU_TRY(cudaMemcpyAsync(c->d_stage_ids, c->h_stage, (size_t)n * 4, cudaMemcpyHostToDevice, st));
+    if (keys16) {
+        memcpy(c->h_stage + (size_t)n * 4, keys16, (size_t)n * 16);
+        CU_TRY(cudaMemcpyAsync(c->d_stage_keys, c->h_stage + (size_t)n * 4, (size_t)n * 16, cudaMemcpyHostToDevice, st));
+    }
+    return GIFT_OK;
+}
+
+int gift_set_keys(gift_ctx* c, const int32_t* user_ids, const uint8_t* keys16, uint32_t n, void* stream)
+{
+    if (!c || (n && (!user_ids || !keys16))) return GIFT_E_INVAL;
+    if (n == 0) return GIFT_OK;
+    DeviceGuard g(c->device);
+    if (!g.ok) return GIFT_E_CUDA;
+    cudaStream_t st = (cudaStream_t)stream;
+    int rc = stage_ids(c, user_ids, keys16, n, st);
+    if (rc != GIFT_OK) return rc;
+    const uint32_t threads = n * POW_LEVELS;
+    key_setup_kernel<<<(threads + 63) / 64, 64, 0, st>>>(c->d_t0, c->d_stage_ids, c->d_stage_keys, n, c->d_hot, c->d_pow);
+    c->launches++;
+    // wipe the staging copies once the kernel has consumed them
+    CU_TRY(cudaMemsetAsync(c->d_stage_keys, 0, (size_t)n * 16, st));
+    CU_TRY(cudaStreamSynchronize(st));
+    memset(c->h_stage, 0, (size_t)n * 20);
+    CU_TRY(cudaGetLastError());
+    return GIFT_OK;
+}
+
+int gift_clear_keys(gift_ctx* c, const int32_t* user_ids, uint32_t n, void* stream)
+{
+    if (!c || (n && !user_ids)) return GIFT_E_INVAL;
+    if (n == 0) return GIFT_OK;
+    DeviceGuard g(c->device);
+    if (!g.ok) return GIFT_E_CUDA;
+    cudaStream_t st = (cudaStream_t)stream;
+    int rc = stage_ids(c, user_ids, nullptr, n, st);
+    if (rc != GIFT_OK) return rc;
+    key_clear_kernel<<<n, 256, 0, st>>>(c->d_stage_ids, n, c->d_hot, c->d_pow);
+    c->launches++;
+    CU_TRY(cudaStreamSynchronize(st));
+    CU_TRY(cudaGetLastError());
+    return GIFT_OK;
+}
+
+int gift_seg_encrypt(gift_ctx* c, const void* src, void* dst, uint64_t buf_bytes, const gift_seg* segs,
+                     uint32_t nseg, const gift_pages* pages, const gift_labels* labels, uint8_t* tags_out,
+                     uint32_t* status, void* stream)
+{
+    return seg_call<MODE_ENCRYPT>(c, src, dst, buf_bytes, segs, nseg, pages, labels, tags_out, status, stream);
+}
+
+int gift_seg_decrypt(gift_ctx* c, const void* src, void* dst, uint64_t buf_bytes, const gift_seg* segs,
+                     uint32_t nseg, const gift_pages* pages, gift_labels* labels, const uint8_t* tags_in,
+                     uint32_t* status, void* stream)
+{
+    return seg_call<MODE_DECRYPT>(c, src, dst, buf_bytes, segs, nseg, pages, labels, (uint8_t*)tags_in, status, stream);
+}
+
+int gift_verify_tags(gift_ctx* c, const void* src, uint64_t buf_bytes, const gift_seg* segs, uint32_t nseg,
+                     const gift_pages* pages, const uint8_t* tags_in, uint32_t* status, void* stream)
+{
+    return seg_call<MODE_VERIFY>(c, src, nullptr, buf_bytes, segs, nseg, pages, nullptr, (uint8_t*)tags_in, status, stream);
+}
+
+int gift_propagate_labels(gift_ctx* c, const gift_rule* rule, const int32_t* const* in_maps, int32_t* out,
+                          uint32_t* viol, void* stream)
+{
+    if (!c || !rule || !in_maps || !viol) return GIFT_E_INVAL;
+    if (rule->n_out && !out) return GIFT_E_INVAL;
+    RuleArgs r;
+    memset(&r, 0, sizeof(r));
+    r.kind = rule->kind; r.n_out = rule->n_out; r.n_in = rule->n_in; r.n_seg = rule->n_seg;
+    r.n_in0 = rule->n_in0; r.n_in1 = rule->n_in1; r.param_mask = rule->param_mask;
+    r.seg_ptr = rule->seg_ptr; r.src_ptr = rule->src_ptr; r.src_idx = rule->src_idx; r.gather = rule->gather;
+    r.out = out; r.viol = viol;
+    uint32_t want_in = 1;
+    switch (rule->kind) {
+    case GIFT_RULE_IDENTITY: break;
+    case GIFT_RULE_BROADCAST: if (!rule->gather && rule->n_out) return GIFT_E_INVAL; break;
+    case GIFT_RULE_ROWWISE:
+        if (rule->n_in < 1 || rule->n_in > 8) return GIFT_E_INVAL;
+        want_in = rule->n_in;
+        break;
+    case GIFT_RULE_SEGREDUCE:
+        if (rule->n_in != 2 || !rule->seg_ptr || !rule->src_ptr || (!rule->src_idx && rule->n_seg)) return GIFT_E_INVAL;
+        want_in = 2;
+        break;
+    default: return GIFT_E_INVAL;
+    }
+    if (rule->n_in != want_in) return GIFT_E_INVAL;
+    for (uint32_t k = 0; k < want_in; k++) {
+        if (!in_maps[k]) return GIFT_E_INVAL;
+        r.in[k] = in_maps[k];
+    }
+    DeviceGuard g(c->device);
+    if (!g.ok) return GIFT_E_CUDA;
+    cudaStream_t st = (cudaStream_t)stream;
+    // Rules read a snapshot: an input that the output overlaps and that is read at other
+    // indices than the one written (the gather source, the block-owner map) is copied first.
+    const int32_t* hazard = nullptr;
+    uint32_t hazard_n = 0, hazard_slot = 0;
+    if (rule->kind == GIFT_RULE_BROADCAST) { hazard = in_maps[0]; hazard_n = rule->n_in0; hazard_slot = 0; }
+    if (rule->kind == GIFT_RULE_SEGREDUCE) { hazard = in_maps[1]; hazard_n = rule->n_in1; hazard_slot = 1; }
+    if (hazard && hazard_n && rule->n_out &&
+        ranges_overlap(hazard, (size_t)hazard_n * 4, out, (size_t)rule->n_out * 4)) {
+        if (hazard_n > c->snapshot_cap) {
+            CU_TRY(cudaDeviceSynchronize());
+            cudaFree(c->d_snapshot);
+            c->d_snapshot = nullptr; c->snapshot_cap = 0;
+            CU_TRY(cudaMalloc(&c->d_snapshot, (size_t)hazard_n * 4));
+            c->snapshot_cap = hazard_n;
+        }
+        CU_TRY(cudaMemcpyAsync(c->d_snapshot, hazard, (size_t)hazard_n * 4, cudaMemcpyDeviceToDevice, st));
+        r.in[hazard_slot] = c->d_snapshot;
+    }
+    viol_init_kernel<<<1, 1, 0, st>>>(viol);
+    c->launches++;
+    if (rule->kind == GIFT_RULE_SEGREDUCE) {
+        const uint64_t threads = (uint64_t)rule->n_seg * 32u + rule->n_out;   // upper bound on uncovered outputs
+        rule_segreduce_kernel<<<(uint32_t)((threads + 255) / 256) + 1, 256, 0, st>>>(r);
+        c->launches++;
+    } else if (rule->n_out) {
+        rule_pointwise_kernel<<<(rule->n_out + 255) / 256, 256, 0, st>>>(r);
+        c->launches++;
+    }
+    CU_TRY(cudaGetLastError());
+    return GIFT_OK;
+}
+
+int gift_timing_enable(gift_ctx* c, int on)
+{
+    if (!c) return GIFT_E_INVAL;
+    DeviceGuard g(c->device);
+    if (!g.ok) return GIFT_E_CUDA;
+    if (on && !c->ev) {
+        c->ev = new (std::nothrow) cudaEvent_t[2 * MAX_TIMED];
+        if (!c->ev) return GIFT_E_NOMEM;
+        for (uint32_t i = 0; i < 2 * MAX_TIMED; i++) {
+            if (cudaEventCreate(&c->ev[i]) != cudaSuccess) {
+                for (uint32_t k = 0; k < i; k++) cudaEventDestroy(c->ev[k]);
+                delete[] c->ev;
+                c->ev = nullptr;
+                return GIFT_E_CUDA;
+            }
+        }
+    }
+    c->timing = on ? 1 : 0;
+    c->n_timed = 0;
+    return GIFT_OK;
+}
+
+int gift_timing_read(gift_ctx* c, double* total_ms, uint32_t* launches)
+{
+    if (!c || !total_ms || !launches) return GIFT_E_INVAL;
+    DeviceGuard g(c->device);
+    if (!g.ok) return GIFT_E_CUDA;
+    double sum = 0.0;
+    for (uint32_t i = 0; i < c->n_timed; i++) {
+        float ms = 0.f;
+        CU_TRY(cudaEventSynchronize(c->ev[2 * i + 1]));
+        CU_TRY(cudaEventElapsedTime(&ms, c->ev[2 * i], c->ev[2 * i + 1]));
+        sum += ms;
+    }
+    *total_ms = sum;
+    *launches = c->n_timed;
+    c->n_timed = 0;
+    return GIFT_OK;
+}
+
+const char* gift_strerror(int code)
+{
+    switch (code) {
+    case GIFT_OK: return "ok";
+    case GIFT_E_INVAL: return "invalid argument";
+    case GIFT_E_NOMEM: return "out of memory";
+    case GIFT_E_CUDA: return "CUDA runtime error";
+    case GIFT_E_RANGE: return "value out of range";
+    case GIFT_E_ALIGN: return "pointer or size not 16-byte aligned";
+    default: return "unknown error";
+    }
+}
+
+uint32_t gift_version(void) { return GIFT_VERSION; }
+
+uint64_t gift_launch_count(const gift_ctx* c) { return c ? c->launches : 0; }
+
+}  // extern "C"

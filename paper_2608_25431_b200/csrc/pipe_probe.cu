@@ -1,0 +1,141 @@
+// Issue-rate probes for the integer, multiply and shared-memory pipes of one SM.
+//
+// The segment cipher is bound by integer instruction throughput, so its roofline
+// needs the per-SM rates of the instructions it is made of.  Each probe runs
+// 1024 threads per SM over long unrolled chains of one instruction kind (eight
+// independent chains per thread hide the latency), times the loop with the SM
+// cycle counter and reports lane-operations per SM clock.
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "../../include/gift.h"
+
+namespace {
+
+constexpr int CHAINS = 8;
+constexpr int UNROLL = 32;
+
+template <int KIND>
+__global__ void __launch_bounds__(1024, 1) probe_kernel(uint32_t iters, uint32_t seed, unsigned long long* cycles,
+                                                        uint32_t* sink)
+{
+    __shared__ uint32_t tab[2048];
+    for (int i = threadIdx.x; i < 2048; i += blockDim.x) tab[i] = (i * 37u + seed) & 2047u & ~31u;
+    __syncthreads();
+    uint32_t x[CHAINS];
+    unsigned long long w[CHAINS];
+#pragma unroll
+    for (int c = 0; c < CHAINS; c++) {
+        x[c] = seed * (c + 1) + threadIdx.x;
+        w[c] = x[c];
+    }
+    const uint32_t k1 = seed | 1u, k2 = seed * 3u + 5u;
+    const uint32_t lane4 = (threadIdx.x & 31u);
+    __syncthreads();
+    const long long t0 = clock64();
+    for (uint32_t it = 0; it < iters; it++) {
+#pragma unroll
+        for (int u = 0; u < UNROLL; u++) {
+#pragma unroll
+            for (int c = 0; c < CHAINS; c++) {
+                if (KIND == 0) {          // three-input logic
+                    asm volatile("lop3.b32 %0, %0, %1, %2, 0x96;" : "+r"(x[c]) : "r"(k1), "r"(k2));
+                } else if (KIND == 1) {   // 32x32+64 -> 64 multiply-add
+                    asm volatile("mad.wide.u32 %0, %1, %2, %0;" : "+l"(w[c]) : "r"(x[c]), "r"(k1));
+                } else if (KIND == 2) {   // byte permute
+                    asm volatile("prmt.b32 %0, %0, %1, 0x2103;" : "+r"(x[c]) : "r"(k1));
+                } else if (KIND == 3) {   // conflict-free shared-memory load, address from the previous load
+                    asm volatile("{ .reg .u32 a; shl.b32 a, %0, 2; ld.shared.u32 %0, [a]; }" : "+r"(x[c]));
+                    (void)lane4;
+                } else if (KIND == 4) {   // funnel shift
+                    asm volatile("shf.l.wrap.b32 %0, %0, %1, 7;" : "+r"(x[c]) : "r"(k1));
+                } else if (KIND == 5) {   // three-input add
+                    asm volatile("add.u32 %0, %0, %1;" : "+r"(x[c]) : "r"(k1));
+                } else if (KIND == 6) {   // logic and wide multiply interleaved: do they share a pipe?
+                    asm volatile("lop3.b32 %0, %0, %1, %2, 0x96;" : "+r"(x[c]) : "r"(k1), "r"(k2));
+                    asm volatile("mad.wide.u32 %0, %1, %2, %0;" : "+l"(w[c]) : "r"(k2), "r"(k1));
+                } else if (KIND == 7) {   // 32x32+32 -> 32 multiply-add (low half)
+                    asm volatile("mad.lo.u32 %0, %0, %1, %2;" : "+r"(x[c]) : "r"(k1), "r"(k2));
+                } else if (KIND == 8) {   // logic and shared-memory loads interleaved
+                    asm volatile("lop3.b32 %0, %0, %1, %2, 0x96;" : "+r"(x[c]) : "r"(k1), "r"(k2));
+                    asm volatile("{ .reg .u32 a; shl.b32 a, %1, 2; ld.shared.u32 %0, [a]; }"
+                                 : "=r"(*reinterpret_cast<uint32_t*>(&w[c])) : "r"(lane4 + (c << 5)));
+                }
+            }
+        }
+    }
+    const long long t1 = clock64();
+    uint32_t acc = 0;
+#pragma unroll
+    for (int c = 0; c < CHAINS; c++) acc ^= x[c] ^ (uint32_t)w[c] ^ (uint32_t)(w[c] >> 32);
+    if (acc == 0x12345678u) sink[0] = acc;     // keeps the chains alive
+    if (threadIdx.x == 0) cycles[blockIdx.x] = (unsigned long long)(t1 - t0);
+    (void)tab;
+}
+
+template <int KIND>
+cudaError_t run_probe(int sms, uint32_t iters, unsigned long long* d_cycles, uint32_t* d_sink, float* ms)
+{
+    cudaEvent_t e0, e1;
+    cudaEventCreate(&e0);
+    cudaEventCreate(&e1);
+    probe_kernel<KIND><<<sms, 1024>>>(4, 12345u, d_cycles, d_sink);        // warm-up
+    cudaEventRecord(e0);
+    probe_kernel<KIND><<<sms, 1024>>>(iters, 12345u, d_cycles, d_sink);
+    cudaEventRecord(e1);
+    cudaError_t e = cudaEventSynchronize(e1);
+    if (e == cudaSuccess) cudaEventElapsedTime(ms, e0, e1);
+    cudaEventDestroy(e0);
+    cudaEventDestroy(e1);
+    return e;
+}
+
+}  // namespace
+
+extern "C" int gift_probe_pipe(int device, int kind, uint32_t iters, double* lane_ops_per_clk_per_sm,
+                               double* sm_mhz)
+{
+    if (!lane_ops_per_clk_per_sm || !sm_mhz || iters == 0 || iters > (1u << 20)) return GIFT_E_INVAL;
+    int prev = -1;
+    if (cudaGetDevice(&prev) != cudaSuccess || cudaSetDevice(device) != cudaSuccess) return GIFT_E_CUDA;
+    cudaDeviceProp prop;
+    if (cudaGetDeviceProperties(&prop, device) != cudaSuccess) return GIFT_E_CUDA;
+    const int sms = prop.multiProcessorCount;
+    unsigned long long* d_cycles = nullptr;
+    uint32_t* d_sink = nullptr;
+    if (cudaMalloc(&d_cycles, sms * sizeof(unsigned long long)) != cudaSuccess) return GIFT_E_NOMEM;
+    if (cudaMalloc(&d_sink, 4) != cudaSuccess) { cudaFree(d_cycles); return GIFT_E_NOMEM; }
+    float ms = 0.f;
+    cudaError_t e;
+    switch (kind) {
+    case 0: e = run_probe<0>(sms, iters, d_cycles, d_sink, &ms); break;
+    case 1: e = run_probe<1>(sms, iters, d_cycles, d_sink, &ms); break;
+    case 2: e = run_probe<2>(sms, iters, d_cycles, d_sink, &ms); break;
+    case 3: e = run_probe<3>(sms, iters, d_cycles, d_sink, &ms); break;
+    case 4: e = run_probe<4>(sms, iters, d_cycles, d_sink, &ms); break;
+    case 5: e = run_probe<5>(sms, iters, d_cycles, d_sink, &ms); break;
+    case 6: e = run_probe<6>(sms, iters, d_cycles, d_sink, &ms); break;
+    case 7: e = run_probe<7>(sms, iters, d_cycles, d_sink, &ms); break;
+    case 8: e = run_probe<8>(sms, iters, d_cycles, d_sink, &ms); break;
+    default: cudaFree(d_cycles); cudaFree(d_sink); cudaSetDevice(prev); return GIFT_E_INVAL;
+    }
+    int rc = GIFT_OK;
+    if (e != cudaSuccess) {
+        rc = GIFT_E_CUDA;
+    } else {
+        unsigned long long* h = new unsigned long long[sms];
+        cudaMemcpy(h, d_cycles, sms * sizeof(unsigned long long), cudaMemcpyDeviceToHost);
+        double mean = 0;
+        for (int i = 0; i < sms; i++) mean += (double)h[i];
+        mean /= sms;
+        delete[] h;
+        const double per_pair = (kind == 6 || kind == 8) ? 2.0 : 1.0;   // two instructions per step
+        const double ops = 1024.0 * CHAINS * UNROLL * (double)iters * per_pair;
+        *lane_ops_per_clk_per_sm = ops / mean;
+        *sm_mhz = mean / (ms * 1e3);
+    }
+    cudaFree(d_cycles);
+    cudaFree(d_sink);
+    cudaSetDevice(prev);
+    return rc;
+}

@@ -1,0 +1,147 @@
+"""Host-side checks that need no GPU: the C-ABI surface, and the device arithmetic compiled
+for the host (field product, table cipher, key schedule, power table and the whole
+run / lane / chain decomposition of a segment) against the CPU oracle."""
+import ctypes as C
+import os
+import re
+
+import numpy as np
+import pytest
+
+from oracle import gcm
+from paper_2608_25431_b200 import build as B
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+def _p(a):
+    return a.ctypes.data_as(C.c_void_p)
+
+
+def _u8(b):
+    return np.frombuffer(bytes(b), dtype=np.uint8).copy()
+
+
+@pytest.fixture(scope="module")
+def hc():
+    return C.CDLL(B.build_hostcheck())
+
+
+def test_library_exports_every_declared_symbol():
+    header = open(os.path.join(ROOT, "include", "gift.h")).read()
+    header = re.sub(r"/\*.*?\*/", "", header, flags=re.S)
+    declared = sorted(set(re.findall(r"\b(gift_[a-z_]+)\s*\(", header)))
+    assert "gift_seg_encrypt" in declared and "gift_propagate_labels" in declared
+    lib = C.CDLL(B.build_lib())          # loading needs no GPU; nothing is called
+    for name in declared:
+        assert hasattr(lib, name), name
+    from paper_2608_25431_b200 import binding
+    assert sorted(binding.EXPORTS) == declared
+
+
+def test_binding_fails_loudly_without_gpu():
+    import torch
+    from paper_2608_25431_b200 import binding
+    if torch.cuda.is_available():
+        pytest.skip("a GPU is present")
+    with pytest.raises(RuntimeError):
+        binding.Ctx(4)
+
+
+def test_t0_table_matches_sbox_definition(hc):
+    t0 = np.zeros(256, dtype=np.uint32)
+    hc.hc_t0_table(_p(t0))
+    s = gcm.sbox().astype(np.uint32)
+    s2 = ((s << 1) ^ np.where(s & 0x80, 0x1B, 0)) & 0xFF
+    assert np.array_equal(t0, s2 | (s << 8) | (s << 16) | ((s2 ^ s) << 24))
+
+
+def test_field_product_matches_oracle(hc):
+    rng = np.random.default_rng(0)
+    special = [bytes(16), b"\x80" + bytes(15), b"\xff" * 16, bytes(15) + b"\x01", b"\x40" + bytes(15)]
+    pairs = [(a, b) for a in special for b in special] + [(rng.bytes(16), rng.bytes(16)) for _ in range(500)]
+    for a, b in pairs:
+        z = np.zeros(16, dtype=np.uint8)
+        hc.hc_gfmul(_p(_u8(a)), _p(_u8(b)), _p(z))
+        assert z.tobytes() == gcm.gf128_mul(a, b)
+
+
+def test_table_cipher_and_key_schedule_match_oracle(hc):
+    rng = np.random.default_rng(1)
+    for _ in range(300):
+        k, b = _u8(rng.bytes(16)), _u8(rng.bytes(16))
+        o = np.zeros(16, dtype=np.uint8)
+        hc.hc_aes_encrypt(_p(k), _p(b), _p(o))
+        assert o.tobytes() == gcm.aes128_encrypt_block(k, b)
+        rk = np.zeros(176, dtype=np.uint8)
+        hc.hc_expand_key(_p(k), _p(rk))
+        assert rk.tobytes() == gcm.key_expand(k).tobytes()
+
+
+def test_power_table_matches_square_and_multiply(hc):
+    rng = np.random.default_rng(2)
+    k = _u8(rng.bytes(16))
+    h = gcm.aes128_encrypt_block(k, bytes(16))
+
+    def power(e):
+        r, b = b"\x80" + bytes(15), h
+        while e:
+            if e & 1:
+                r = gcm.gf128_mul(r, b)
+            b = gcm.gf128_mul(b, b)
+            e >>= 1
+        return r
+
+    for e in [0, 1, 2, 31, 32, 33, 255, 256, 257, 65535, 65536, 1 << 24, (1 << 32) - 1, 123456789]:
+        o = np.zeros(16, dtype=np.uint8)
+        hc.hc_power(_p(k), C.c_uint64(e), _p(o))
+        assert o.tobytes() == power(e), e
+
+
+@pytest.mark.parametrize("chains", [1, 2])
+def test_run_decomposition_reproduces_gcm(hc, chains):
+    """Every (length, run length) split of a segment into runs, lanes and chains gives the oracle's bytes and tag."""
+    rng = np.random.default_rng(3 + chains)
+    for n in [0, 1, 15, 16, 17, 31, 32, 33, 511, 512, 513, 1024, 1040, 2048 + 7, 4096, 5000, 70000]:
+        for run_blocks in (32, 64, 96, 1024):
+            k, nonce = _u8(rng.bytes(16)), _u8(rng.bytes(12))
+            pt = _u8(rng.bytes(n + 32))
+            ct = np.full(n + 32, 0xEE, dtype=np.uint8)
+            tag = np.zeros(16, dtype=np.uint8)
+            hc.hc_segment(_p(k), _p(nonce), _p(pt), _p(ct), None, C.c_uint64(0), C.c_uint64(16), C.c_uint64(n),
+                          C.c_uint32(run_blocks), chains, 0, _p(tag))
+            ref_ct, ref_tag = gcm.gcm_encrypt(k, nonce, pt[16:16 + n])
+            assert ct[16:16 + n].tobytes() == ref_ct and tag.tobytes() == ref_tag, (n, run_blocks)
+            assert (ct[:16] == 0xEE).all() and (ct[16 + n:] == 0xEE).all()      # nothing outside the segment
+            out = np.full(n + 32, 0xEE, dtype=np.uint8)
+            tag2 = np.zeros(16, dtype=np.uint8)
+            hc.hc_segment(_p(k), _p(nonce), _p(ct), _p(out), None, C.c_uint64(0), C.c_uint64(16), C.c_uint64(n),
+                          C.c_uint32(run_blocks), chains, 1, _p(tag2))
+            assert out[16:16 + n].tobytes() == pt[16:16 + n].tobytes() and tag2.tobytes() == ref_tag
+            tag3 = np.zeros(16, dtype=np.uint8)
+            hc.hc_segment(_p(k), _p(nonce), _p(ct), _p(out), None, C.c_uint64(0), C.c_uint64(16), C.c_uint64(n),
+                          C.c_uint32(run_blocks), chains, 2, _p(tag3))
+            assert tag3.tobytes() == ref_tag
+
+
+def test_paged_addressing_reproduces_gcm(hc):
+    rng = np.random.default_rng(9)
+    pb = 160
+    for n in [100, 160, 161, 1000, 3000, 3200]:
+        npg = (n + pb - 1) // pb
+        table = rng.permutation(40).astype(np.int32)
+        buf = _u8(rng.bytes(40 * pb))
+        out = buf.copy()
+        tag = np.zeros(16, dtype=np.uint8)
+        k, nonce = _u8(rng.bytes(16)), _u8(rng.bytes(12))
+        hc.hc_segment(_p(k), _p(nonce), _p(buf), _p(out), _p(table), C.c_uint64(pb), C.c_uint64(3), C.c_uint64(n),
+                      C.c_uint32(64), 2, 0, _p(tag))
+        sl = [(int(table[3 + i]) * pb, min(pb, n - i * pb)) for i in range(npg)]
+        plain = b"".join(buf[o:o + l].tobytes() for o, l in sl)
+        got = b"".join(out[o:o + l].tobytes() for o, l in sl)
+        ref_ct, ref_tag = gcm.gcm_encrypt(k, nonce, plain)
+        assert got == ref_ct and tag.tobytes() == ref_tag, n
+        touched = np.zeros(40 * pb, dtype=bool)
+        for o, l in sl:
+            touched[o:o + l] = True
+        assert np.array_equal(out[~touched], buf[~touched])
