@@ -48,6 +48,7 @@ struct gift_ctx {
     uint32_t flags;
     int chains;                        // Horner chains per lane (1 or 2)
     int tables;                        // T-tables held in shared memory (2 or 4)
+    int threads;                       // threads per CTA of the cipher kernel (512 or 1024)
     int num_sms;
     uint32_t* d_t0;                    // 256-entry T0 in global memory
     KeyHot* d_hot;                     // [max_users]
@@ -356,8 +357,8 @@ __device__ __forceinline__ uint32_t warp_xor(uint32_t v)
     return v;
 }
 
-template <int U, int MODE, int NT>
-__global__ void __launch_bounds__(512, 1) crypt_kernel(CallArgs a, const uint32_t* __restrict__ t0)
+template <int U, int MODE, int NT, int THREADS>
+__global__ void __launch_bounds__(THREADS, 1) crypt_kernel(CallArgs a, const uint32_t* __restrict__ t0)
 {
     constexpr uint32_t TAB_BYTES = NT == 4 ? 131072u : 65536u;
     const int lane = threadIdx.x & 31, wid = threadIdx.x >> 5;
@@ -651,17 +652,12 @@ int ensure_scratch(gift_ctx* c, uint32_t nseg)
     return GIFT_OK;
 }
 
-size_t crypt_smem_bytes(int tables)
-{
-    return (tables == 4 ? 131072u : 65536u) + 16u * sizeof(KeyHot);
-}
-
-template <int U, int MODE, int NT>
+template <int U, int MODE, int NT, int THREADS>
 int launch_crypt_t(gift_ctx* c, const CallArgs& a, cudaStream_t st)
 {
-    const size_t smem = crypt_smem_bytes(NT);
+    const size_t smem = (NT == 4 ? 131072u : 65536u) + (THREADS / 32) * sizeof(KeyHot);
     static bool configured[8] = {false, false, false, false, false, false, false, false};
-    auto kern = crypt_kernel<U, MODE, NT>;
+    auto kern = crypt_kernel<U, MODE, NT, THREADS>;
     if (c->device < 8 && !configured[c->device]) {
         CU_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
         configured[c->device] = true;
@@ -670,7 +666,7 @@ int launch_crypt_t(gift_ctx* c, const CallArgs& a, cudaStream_t st)
     }
     const bool timed = c->timing && c->ev && c->n_timed < MAX_TIMED;
     if (timed) CU_TRY(cudaEventRecord(c->ev[2 * c->n_timed], st));
-    kern<<<c->num_sms, 512, smem, st>>>(a, c->d_t0);
+    kern<<<c->num_sms, THREADS, smem, st>>>(a, c->d_t0);
     if (timed) {
         CU_TRY(cudaEventRecord(c->ev[2 * c->n_timed + 1], st));
         c->n_timed++;
@@ -682,10 +678,14 @@ int launch_crypt_t(gift_ctx* c, const CallArgs& a, cudaStream_t st)
 template <int MODE>
 int launch_crypt(gift_ctx* c, const CallArgs& a, cudaStream_t st)
 {
-    if (c->tables == 4) {
-        return c->chains == 2 ? launch_crypt_t<2, MODE, 4>(c, a, st) : launch_crypt_t<1, MODE, 4>(c, a, st);
+    if (c->threads == 1024) {
+        if (c->tables == 4) return launch_crypt_t<1, MODE, 4, 1024>(c, a, st);
+        return launch_crypt_t<1, MODE, 2, 1024>(c, a, st);
     }
-    return c->chains == 2 ? launch_crypt_t<2, MODE, 2>(c, a, st) : launch_crypt_t<1, MODE, 2>(c, a, st);
+    if (c->tables == 4) {
+        return c->chains == 2 ? launch_crypt_t<2, MODE, 4, 512>(c, a, st) : launch_crypt_t<1, MODE, 4, 512>(c, a, st);
+    }
+    return c->chains == 2 ? launch_crypt_t<2, MODE, 2, 512>(c, a, st) : launch_crypt_t<1, MODE, 2, 512>(c, a, st);
 }
 
 template <int MODE>
@@ -723,7 +723,7 @@ int seg_call(gift_ctx* c, const void* src, void* dst, uint64_t buf_bytes, const 
     a.acc = c->d_acc;
     a.ticket = c->d_ticket;
     a.glob = c->d_glob;
-    a.target_runs = (uint32_t)c->num_sms * 16u * 8u;     // about eight runs per resident warp
+    a.target_runs = (uint32_t)c->num_sms * (uint32_t)(c->threads / 32) * 8u;   // about eight runs per resident warp
     a.max_run_blocks = 4096u;                             // 64 KiB
     a.min_run_blocks = 256u;                              // 4 KiB
 
@@ -761,10 +761,13 @@ int gift_ctx_create(gift_ctx** out, int device, uint32_t max_users, uint32_t fla
 {
     if (!out || max_users == 0) return GIFT_E_INVAL;
     *out = nullptr;
-    int chains = (int)(flags & 0xFu), tables = (int)((flags >> 4) & 0xFu);
-    if (chains == 0) chains = 2;
+    int chains = (int)(flags & 0xFu), tables = (int)((flags >> 4) & 0xFu), threads = (int)((flags >> 8) & 0xFu) * 512;
+    if (chains == 0) chains = 1;
     if (tables == 0) tables = 4;
-    if ((chains != 1 && chains != 2) || (tables != 2 && tables != 4) || (flags >> 8)) return GIFT_E_INVAL;
+    if (threads == 0) threads = 512;
+    if ((chains != 1 && chains != 2) || (tables != 2 && tables != 4) || (threads != 512 && threads != 1024) ||
+        (threads == 1024 && chains != 1) || (flags >> 12))
+        return GIFT_E_INVAL;
     if (max_users > (1u << 20)) return GIFT_E_RANGE;
     DeviceGuard g(device);
     if (!g.ok) return GIFT_E_CUDA;
@@ -776,6 +779,7 @@ int gift_ctx_create(gift_ctx** out, int device, uint32_t max_users, uint32_t fla
     c->flags = flags;
     c->chains = chains;
     c->tables = tables;
+    c->threads = threads;
     int rc = GIFT_OK;
     cudaDeviceProp prop;
     if (cudaGetDeviceProperties(&prop, device) != cudaSuccess) { delete c; return GIFT_E_CUDA; }

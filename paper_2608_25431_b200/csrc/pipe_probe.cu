@@ -19,14 +19,18 @@ template <int KIND>
 __global__ void __launch_bounds__(1024, 1) probe_kernel(uint32_t iters, uint32_t seed, unsigned long long* cycles,
                                                         uint32_t* sink)
 {
+    // tab[i] is a multiple of 32 below 2048, so tab[tab[i] + lane] stays inside the table and
+    // every lane of a warp reads its own bank
     __shared__ uint32_t tab[2048];
-    for (int i = threadIdx.x; i < 2048; i += blockDim.x) tab[i] = (i * 37u + seed) & 2047u & ~31u;
+    for (int i = threadIdx.x; i < 2048; i += blockDim.x) tab[i] = ((i >> 5) * 37u + seed) & 2047u & ~31u;
     __syncthreads();
+    const volatile uint32_t* vtab = tab;
     uint32_t x[CHAINS];
     unsigned long long w[CHAINS];
 #pragma unroll
     for (int c = 0; c < CHAINS; c++) {
         x[c] = seed * (c + 1) + threadIdx.x;
+        if (KIND == 3) x[c] = (x[c] & 2047u & ~31u);
         w[c] = x[c];
     }
     const uint32_t k1 = seed | 1u, k2 = seed * 3u + 5u;
@@ -45,8 +49,7 @@ __global__ void __launch_bounds__(1024, 1) probe_kernel(uint32_t iters, uint32_t
                 } else if (KIND == 2) {   // byte permute
                     asm volatile("prmt.b32 %0, %0, %1, 0x2103;" : "+r"(x[c]) : "r"(k1));
                 } else if (KIND == 3) {   // conflict-free shared-memory load, address from the previous load
-                    asm volatile("{ .reg .u32 a; shl.b32 a, %0, 2; ld.shared.u32 %0, [a]; }" : "+r"(x[c]));
-                    (void)lane4;
+                    x[c] = vtab[x[c] + lane4];
                 } else if (KIND == 4) {   // funnel shift
                     asm volatile("shf.l.wrap.b32 %0, %0, %1, 7;" : "+r"(x[c]) : "r"(k1));
                 } else if (KIND == 5) {   // three-input add
@@ -56,10 +59,36 @@ __global__ void __launch_bounds__(1024, 1) probe_kernel(uint32_t iters, uint32_t
                     asm volatile("mad.wide.u32 %0, %1, %2, %0;" : "+l"(w[c]) : "r"(k2), "r"(k1));
                 } else if (KIND == 7) {   // 32x32+32 -> 32 multiply-add (low half)
                     asm volatile("mad.lo.u32 %0, %0, %1, %2;" : "+r"(x[c]) : "r"(k1), "r"(k2));
+                } else if (KIND == 9) {   // 32x32 -> 64 multiply without accumulate
+                    asm volatile("mul.wide.u32 %0, %1, %2;" : "=l"(w[c]) : "r"(x[c]), "r"(k1));
+                } else if (KIND == 10) {  // logic + wide multiply without accumulate
+                    asm volatile("lop3.b32 %0, %0, %1, %2, 0x96;" : "+r"(x[c]) : "r"(k1), "r"(k2));
+                    asm volatile("mul.wide.u32 %0, %1, %2;" : "=l"(w[c]) : "r"(k2), "r"(k1));
+                } else if (KIND == 11) {  // logic + 32-bit multiply-add
+                    asm volatile("lop3.b32 %0, %0, %1, %2, 0x96;" : "+r"(x[c]) : "r"(k1), "r"(k2));
+                    asm volatile("mad.lo.u32 %0, %1, %2, %3;" : "=r"(*reinterpret_cast<uint32_t*>(&w[c])) : "r"(k2), "r"(k1), "r"(k2));
+                } else if (KIND == 12) {  // logic + add
+                    asm volatile("lop3.b32 %0, %0, %1, %2, 0x96;" : "+r"(x[c]) : "r"(k1), "r"(k2));
+                    asm volatile("add.u32 %0, %1, %2;" : "=r"(*reinterpret_cast<uint32_t*>(&w[c])) : "r"(k2), "r"(k1));
+                } else if (KIND == 13) {  // byte permute + wide multiply-add
+                    asm volatile("prmt.b32 %0, %0, %1, 0x2103;" : "+r"(x[c]) : "r"(k1));
+                    asm volatile("mad.wide.u32 %0, %1, %2, %0;" : "+l"(w[c]) : "r"(k2), "r"(k1));
+                } else if (KIND == 14) {  // logic with an immediate operand + wide multiply-add
+                    asm volatile("lop3.b32 %0, %0, %1, 0x11111111, 0x96;" : "+r"(x[c]) : "r"(k1));
+                    asm volatile("mad.wide.u32 %0, %1, %2, %0;" : "+l"(w[c]) : "r"(k2), "r"(k1));
+                } else if (KIND == 15) {  // two logic + one wide multiply-add
+                    asm volatile("lop3.b32 %0, %0, %1, %2, 0x96;" : "+r"(x[c]) : "r"(k1), "r"(k2));
+                    asm volatile("lop3.b32 %0, %0, %1, %2, 0x69;" : "+r"(x[c]) : "r"(k2), "r"(k1));
+                    asm volatile("mad.wide.u32 %0, %1, %2, %0;" : "+l"(w[c]) : "r"(k2), "r"(k1));
+                } else if (KIND == 16) {  // shared load + wide multiply-add
+                    w[c] += vtab[lane4 + (c << 5)];
+                    asm volatile("mad.wide.u32 %0, %1, %2, %0;" : "+l"(w[c]) : "r"(k2), "r"(k1));
+                } else if (KIND == 17) {  // logic + permute (both integer pipe)
+                    asm volatile("lop3.b32 %0, %0, %1, %2, 0x96;" : "+r"(x[c]) : "r"(k1), "r"(k2));
+                    asm volatile("prmt.b32 %0, %0, %1, 0x2103;" : "+r"(x[c]) : "r"(k1));
                 } else if (KIND == 8) {   // logic and shared-memory loads interleaved
                     asm volatile("lop3.b32 %0, %0, %1, %2, 0x96;" : "+r"(x[c]) : "r"(k1), "r"(k2));
-                    asm volatile("{ .reg .u32 a; shl.b32 a, %1, 2; ld.shared.u32 %0, [a]; }"
-                                 : "=r"(*reinterpret_cast<uint32_t*>(&w[c])) : "r"(lane4 + (c << 5)));
+                    w[c] = vtab[lane4 + (c << 5)];
                 }
             }
         }
@@ -70,7 +99,6 @@ __global__ void __launch_bounds__(1024, 1) probe_kernel(uint32_t iters, uint32_t
     for (int c = 0; c < CHAINS; c++) acc ^= x[c] ^ (uint32_t)w[c] ^ (uint32_t)(w[c] >> 32);
     if (acc == 0x12345678u) sink[0] = acc;     // keeps the chains alive
     if (threadIdx.x == 0) cycles[blockIdx.x] = (unsigned long long)(t1 - t0);
-    (void)tab;
 }
 
 template <int KIND>
@@ -117,6 +145,15 @@ extern "C" int gift_probe_pipe(int device, int kind, uint32_t iters, double* lan
     case 6: e = run_probe<6>(sms, iters, d_cycles, d_sink, &ms); break;
     case 7: e = run_probe<7>(sms, iters, d_cycles, d_sink, &ms); break;
     case 8: e = run_probe<8>(sms, iters, d_cycles, d_sink, &ms); break;
+    case 9: e = run_probe<9>(sms, iters, d_cycles, d_sink, &ms); break;
+    case 10: e = run_probe<10>(sms, iters, d_cycles, d_sink, &ms); break;
+    case 11: e = run_probe<11>(sms, iters, d_cycles, d_sink, &ms); break;
+    case 12: e = run_probe<12>(sms, iters, d_cycles, d_sink, &ms); break;
+    case 13: e = run_probe<13>(sms, iters, d_cycles, d_sink, &ms); break;
+    case 14: e = run_probe<14>(sms, iters, d_cycles, d_sink, &ms); break;
+    case 15: e = run_probe<15>(sms, iters, d_cycles, d_sink, &ms); break;
+    case 16: e = run_probe<16>(sms, iters, d_cycles, d_sink, &ms); break;
+    case 17: e = run_probe<17>(sms, iters, d_cycles, d_sink, &ms); break;
     default: cudaFree(d_cycles); cudaFree(d_sink); cudaSetDevice(prev); return GIFT_E_INVAL;
     }
     int rc = GIFT_OK;
@@ -129,7 +166,8 @@ extern "C" int gift_probe_pipe(int device, int kind, uint32_t iters, double* lan
         for (int i = 0; i < sms; i++) mean += (double)h[i];
         mean /= sms;
         delete[] h;
-        const double per_pair = (kind == 6 || kind == 8) ? 2.0 : 1.0;   // two instructions per step
+        static const double per_step[18] = {1, 1, 1, 1, 1, 1, 2, 1, 2, 1, 2, 2, 2, 2, 2, 3, 2, 2};
+        const double per_pair = per_step[kind];                       // instructions per step
         const double ops = 1024.0 * CHAINS * UNROLL * (double)iters * per_pair;
         *lane_ops_per_clk_per_sm = ops / mean;
         *sm_mhz = mean / (ms * 1e3);
