@@ -143,6 +143,30 @@ int gift_seg_encrypt(gift_ctx* ctx, const void* src, void* dst, uint64_t buf_byt
                      const gift_seg* segs, uint32_t nseg, const gift_pages* pages,
                      const gift_labels* labels, uint8_t* tags_out, uint32_t* status, void* stream);
 
+/* gift_seg_encrypt for callers that are not allowed to allocate device memory (the paper
+ * has no counterpart; it is an addition of this library).  Some hosts of this code cannot
+ * call cudaMalloc at the point where they export data: a serving loop that has handed all
+ * device memory to its own pool, a plugin that runs under a framework's allocator, code
+ * that runs where an allocation would stall every stream.  gift_seg_encrypt grows its
+ * scratch with cudaMalloc when a call has more segments than any before it; this entry
+ * point never does.  It calls no cudaMalloc, cudaFree or other allocating routine: its
+ * scratch (work list, partial hashes, counters) is a fixed array inside the library image,
+ * about 1.6 MB, which every GPU that loads the library holds until the process exits.
+ *   - Arguments, results and status words are exactly those of gift_seg_encrypt; the ctx
+ *     (created earlier, when allocation was still allowed) supplies the keys.
+ *   - nseg must not exceed GIFT_STATIC_MAX_SEGS (65536); a larger table is refused with
+ *     GIFT_E_RANGE and nothing is launched.
+ *   - The first call on a device looks up the array's device address; make that first
+ *     call before any stream capture begins.
+ *   - All calls on one GPU share the array.  Each call clears what it needs, so calls may
+ *     follow one another freely on one stream, but two calls whose kernels can overlap on
+ *     the GPU (different streams, different ctxs, different threads) race on it and give
+ *     wrong tags.  Serialise them, or use gift_seg_encrypt for the concurrent ones. */
+#define GIFT_STATIC_MAX_SEGS 65536u
+int gift_seg_encrypt_static(gift_ctx* ctx, const void* src, void* dst, uint64_t buf_bytes,
+                            const gift_seg* segs, uint32_t nseg, const gift_pages* pages,
+                            const gift_labels* labels, uint8_t* tags_out, uint32_t* status, void* stream);
+
 /* Import (paper sec. 3 steps 3-4): decrypt each segment with the CLAIMED
  * owner's key after checking tags_in[i] over the received ciphertext.  On a
  * match dst receives the plaintext and, if labels are given, the covered units

@@ -19,10 +19,12 @@ OK, E_INVAL, E_NOMEM, E_CUDA, E_RANGE, E_ALIGN = 0, -1, -2, -3, -4, -5
 ST_TAG_MISMATCH, ST_OWNER_MISMATCH, ST_UNOWNED, ST_NO_KEY, ST_BAD_DESC = 1, 2, 4, 8, 16
 OWNER_PARAM, OWNER_NONE, OWNER_CONFLICT = -1, -2, -3
 RULE_IDENTITY, RULE_ROWWISE, RULE_SEGREDUCE, RULE_BROADCAST = 0, 1, 2, 3
+STATIC_MAX_SEGS = 65536
 
 EXPORTS = [
     "gift_ctx_create", "gift_ctx_destroy", "gift_ctx_reserve", "gift_set_keys", "gift_clear_keys",
-    "gift_seg_encrypt", "gift_seg_decrypt", "gift_verify_tags", "gift_propagate_labels",
+    "gift_seg_encrypt", "gift_seg_encrypt_static", "gift_seg_decrypt", "gift_verify_tags",
+    "gift_propagate_labels",
     "gift_strerror", "gift_version", "gift_launch_count", "gift_timing_enable", "gift_timing_read",
     "gift_probe_pipe",
 ]
@@ -68,6 +70,7 @@ def lib():
         l.gift_seg_encrypt.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_uint64, C.c_void_p, C.c_uint32,
                                        C.POINTER(_Pages), C.POINTER(_Labels), C.c_void_p, C.c_void_p, C.c_void_p]
         l.gift_seg_decrypt.argtypes = l.gift_seg_encrypt.argtypes
+        l.gift_seg_encrypt_static.argtypes = l.gift_seg_encrypt.argtypes
         l.gift_verify_tags.argtypes = [C.c_void_p, C.c_void_p, C.c_uint64, C.c_void_p, C.c_uint32,
                                        C.POINTER(_Pages), C.c_void_p, C.c_void_p, C.c_void_p]
         l.gift_propagate_labels.argtypes = [C.c_void_p, C.POINTER(_Rule), C.POINTER(C.c_void_p), C.c_void_p,
@@ -173,6 +176,19 @@ class Ctx:
         _check(lib().gift_seg_encrypt(self._h, _dev(src), _dev(dst), src.numel() * src.element_size(), _dev(segs),
                                       nseg, C.byref(pg) if pg else None, C.byref(lb) if lb else None,
                                       _dev(tags_out), _dev(status), _stream_ptr(stream)), "gift_seg_encrypt")
+
+    def seg_encrypt_static(self, src, dst, segs, nseg, tags_out, status, page_table=None, page_bytes=0,
+                           owner_map=None, unit_bytes=0, stream=None):
+        """gift_seg_encrypt_static: same results as seg_encrypt, but allocates nothing.
+
+        For callers that cannot call cudaMalloc when they export data; at most
+        STATIC_MAX_SEGS segments per call, and calls that overlap on the GPU race on the
+        library's fixed scratch array (see include/gift.h)."""
+        pg, lb = self._tables(page_table, page_bytes, owner_map, unit_bytes)
+        _check(lib().gift_seg_encrypt_static(self._h, _dev(src), _dev(dst), src.numel() * src.element_size(),
+                                             _dev(segs), nseg, C.byref(pg) if pg else None,
+                                             C.byref(lb) if lb else None, _dev(tags_out), _dev(status),
+                                             _stream_ptr(stream)), "gift_seg_encrypt_static")
 
     def seg_decrypt(self, src, dst, segs, nseg, tags_in, status, page_table=None, page_bytes=0,
                     owner_map=None, unit_bytes=0, stream=None):

@@ -1040,3 +1040,101 @@ uint32_t gift_version(void) { return GIFT_VERSION; }
 uint64_t gift_launch_count(const gift_ctx* c) { return c ? c->launches : 0; }
 
 }  // extern "C"
+
+// ---------------------------------------------------------------------------
+// gift_seg_encrypt_static: the export call for callers that must not allocate
+// ---------------------------------------------------------------------------
+//
+// Same kernels as gift_seg_encrypt, but the per-call scratch (work list, partial
+// hashes, tickets, counters) lives in one file-scope device array instead of
+// memory the ctx grows with cudaMalloc.  The array belongs to the loaded library:
+// every GPU that loads libgift.so holds GIFT_STATIC_SCRATCH_BYTES of it until the
+// process exits, and every call on that GPU shares it.
+
+#define GIFT_STATIC_MAX_SEGS 65536u
+
+namespace {
+
+constexpr size_t STATIC_OFF_PREFIX = 256;                                                   // after Globals
+constexpr size_t STATIC_OFF_ACC = STATIC_OFF_PREFIX + ((size_t)GIFT_STATIC_MAX_SEGS + 64) * 4;   // 16-byte aligned
+constexpr size_t STATIC_OFF_TICKET = STATIC_OFF_ACC + (size_t)GIFT_STATIC_MAX_SEGS * 16;
+constexpr size_t STATIC_SCRATCH_BYTES = STATIC_OFF_TICKET + (size_t)GIFT_STATIC_MAX_SEGS * 4;
+static_assert(sizeof(Globals) <= STATIC_OFF_PREFIX && STATIC_OFF_ACC % 16 == 0, "static scratch layout");
+
+// In host code this name is only a handle for the symbol, never a device address:
+// the address a kernel can use comes from cudaGetSymbolAddress, per device.
+static __device__ __align__(256) unsigned char g_static_scratch[STATIC_SCRATCH_BYTES];
+
+constexpr int STATIC_MAX_DEVICES = 64;
+unsigned char* g_static_ptr[STATIC_MAX_DEVICES];      // device address of the array on each GPU, once known
+
+// First use on a device: look the symbol up with that device current.
+int static_scratch_for(int device, unsigned char** out)
+{
+    if (device < 0 || device >= STATIC_MAX_DEVICES) return GIFT_E_RANGE;
+    if (g_static_ptr[device] == nullptr) {
+        void* p = nullptr;
+        const cudaError_t e = cudaGetSymbolAddress(&p, g_static_scratch);
+        if (e != cudaSuccess || p == nullptr) return GIFT_E_CUDA;
+        g_static_ptr[device] = static_cast<unsigned char*>(p);
+    }
+    *out = g_static_ptr[device];
+    return GIFT_OK;
+}
+
+}  // namespace
+
+extern "C" int gift_seg_encrypt_static(gift_ctx* c, const void* src, void* dst, uint64_t buf_bytes,
+                                       const gift_seg* segs, uint32_t nseg, const gift_pages* pages,
+                                       const gift_labels* labels, uint8_t* tags_out, uint32_t* status,
+                                       void* stream)
+{
+    if (!c || !segs || !tags_out || !status) return nseg == 0 && c ? GIFT_OK : GIFT_E_INVAL;
+    if (nseg == 0) return GIFT_OK;
+    if (nseg > GIFT_STATIC_MAX_SEGS) return GIFT_E_RANGE;     // larger tables need gift_seg_encrypt
+    if (!src || !dst) return GIFT_E_INVAL;
+    if (((uintptr_t)src & 15) || ((uintptr_t)dst & 15) || ((uintptr_t)tags_out & 15)) return GIFT_E_ALIGN;
+    if (pages && (!pages->table || pages->page_bytes == 0)) return GIFT_E_INVAL;
+    if (pages && (pages->page_bytes & 15)) return GIFT_E_ALIGN;
+    if (labels && (!labels->owner_map || (!pages && labels->unit_bytes == 0))) return GIFT_E_INVAL;
+    DeviceGuard g(c->device);
+    if (!g.ok) return GIFT_E_CUDA;
+    unsigned char* scratch = nullptr;
+    const int rc0 = static_scratch_for(c->device, &scratch);
+    if (rc0 != GIFT_OK) return rc0;
+    cudaStream_t st = (cudaStream_t)stream;
+
+    CallArgs a;
+    memset(&a, 0, sizeof(a));
+    a.src = (const uint8_t*)src;
+    a.dst = (uint8_t*)dst;
+    a.buf_bytes = buf_bytes;
+    a.segs = segs;
+    a.nseg = nseg;
+    if (pages) { a.page_table = pages->table; a.n_pages = pages->n; a.page_bytes = pages->page_bytes; }
+    if (labels) { a.owner_map = labels->owner_map; a.n_units = labels->n_units; a.unit_bytes = labels->unit_bytes; }
+    a.tags = tags_out;
+    a.status = status;
+    a.hot = c->d_hot;
+    a.pow = c->d_pow;
+    a.max_users = c->max_users;
+    a.glob = reinterpret_cast<Globals*>(scratch);
+    a.run_prefix = reinterpret_cast<uint32_t*>(scratch + STATIC_OFF_PREFIX);
+    a.acc = reinterpret_cast<uint4*>(scratch + STATIC_OFF_ACC);
+    a.ticket = reinterpret_cast<uint32_t*>(scratch + STATIC_OFF_TICKET);
+    a.target_runs = (uint32_t)c->num_sms * (uint32_t)(c->threads / 32) * 8u;
+    a.max_run_blocks = 4096u;
+    a.min_run_blocks = 256u;
+
+    // The array still holds the previous call's values: the counters are cleared here, the
+    // per-segment accumulators and tickets by the plan kernel, the work list by the scan kernel.
+    CU_TRY(cudaMemsetAsync(a.glob, 0, sizeof(Globals), st));
+    plan_kernel<MODE_ENCRYPT><<<(nseg + 7) / 8, 256, 0, st>>>(a);
+    scan_kernel<<<1, 1024, 0, st>>>(a);
+    c->launches += 2;
+    const int rc = launch_crypt<MODE_ENCRYPT>(c, a, st);
+    if (rc != GIFT_OK) return rc;
+    CU_TRY(cudaGetLastError());
+    return GIFT_OK;
+}
+
