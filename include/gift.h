@@ -106,10 +106,12 @@ typedef struct {
 /* Create a context on CUDA device `device` able to hold keys for user ids
  * 0 .. max_users-1 (about 17 KiB of device memory per user: round keys and
  * powers of the hash subkey), max_users <= 2^20.  flags selects a kernel
- * variant: 0 for the default, else GIFT_CTX_FLAGS(tables, chains) with tables
+ * variant: 0 for the default, else GIFT_CTX_FLAGS(threads, tables, chains) with
+ * threads in {0, 512, 768, 1024} (cipher-kernel CTA size, 0 = default), tables
  * in {2, 4} (T-tables kept in shared memory) and chains in {1, 2} (hash chains
- * per lane); every variant computes the same results.  Host call; synchronises. */
-#define GIFT_CTX_FLAGS(tables, chains)  ((uint32_t)(((tables) << 4) | (chains)))
+ * per lane; 2 needs 512 threads); every variant computes the same results.
+ * Host call; synchronises. */
+#define GIFT_CTX_FLAGS(threads, tables, chains)  ((uint32_t)((((threads) / 256) << 8) | ((tables) << 4) | (chains)))
 int gift_ctx_create(gift_ctx** out, int device, uint32_t max_users, uint32_t flags);
 
 /* Zero all key material on the device and free the ctx.  Synchronises. */

@@ -66,6 +66,39 @@ GIFT_HD uint64_t mulwide(uint32_t a, uint32_t b)
     return (uint64_t)a * (uint64_t)b;
 }
 
+// Small multipliers (1, 2, 4, 128) that the compiler cannot see through.  On this GPU
+// logic, permute and shift instructions share one pipe, which binds the cipher kernel,
+// while the multiply pipe is mostly idle.  An add written as a*1 + b, or a shift written
+// as a 32x32 -> 64 multiply by 2^s, stays a multiply instruction only if the factor is
+// not a compile-time constant; constant memory that the host could rewrite is opaque
+// enough.  The values never change.
+#if defined(__CUDACC__)
+__constant__ uint32_t gift_kmul[4] = {1u, 2u, 4u, 128u};
+#endif
+static const uint32_t gift_kmul_host[4] = {1u, 2u, 4u, 128u};
+#if defined(__CUDA_ARCH__)
+#define GIFT_KMUL(i) gift_kmul[i]
+#else
+#define GIFT_KMUL(i) gift_kmul_host[i]
+#endif
+
+#ifndef GIFT_ADD_ON_MUL
+#define GIFT_ADD_ON_MUL 1
+#endif
+#ifndef GIFT_REDUCE_ON_MUL
+#define GIFT_REDUCE_ON_MUL 0
+#endif
+
+// a + b on the multiply pipe
+GIFT_HD uint32_t add_mul(uint32_t a, uint32_t b)
+{
+#if GIFT_ADD_ON_MUL
+    return a * GIFT_KMUL(0) + b;
+#else
+    return a + b;
+#endif
+}
+
 // Reverse the bits inside each byte of a little-endian word: block bytes <-> natural domain.
 GIFT_HD uint32_t reflect_bytes(uint32_t x)
 {
@@ -116,13 +149,22 @@ GIFT_HD split32 split_word(uint32_t b)
 GIFT_HD uint64_t clmul32(uint32_t a, const split32& b)
 {
     const uint32_t a0 = a & GIFT_M0, a1 = a & GIFT_M1, a2 = a & GIFT_M2, a3 = a & GIFT_M3;
-    // class r collects the products a_i * b_j with i + j == r (mod 4)
-    uint64_t c0 = mulwide(a0, b.m[0]) ^ mulwide(a1, b.m[3]) ^ mulwide(a2, b.m[2]) ^ mulwide(a3, b.m[1]);
-    uint64_t c1 = mulwide(a0, b.m[1]) ^ mulwide(a1, b.m[0]) ^ mulwide(a2, b.m[3]) ^ mulwide(a3, b.m[2]);
-    uint64_t c2 = mulwide(a0, b.m[2]) ^ mulwide(a1, b.m[1]) ^ mulwide(a2, b.m[0]) ^ mulwide(a3, b.m[3]);
-    uint64_t c3 = mulwide(a0, b.m[3]) ^ mulwide(a1, b.m[2]) ^ mulwide(a2, b.m[1]) ^ mulwide(a3, b.m[0]);
-    return (c0 & 0x1111111111111111ull) | (c1 & 0x2222222222222222ull) |
-           (c2 & 0x4444444444444444ull) | (c3 & 0x8888888888888888ull);
+    // class r collects the products a_i * b_j with i + j == r (mod 4).  The four masked
+    // classes occupy disjoint bits, so they are merged with integer adds, issued as
+    // multiply-adds to keep them off the logic pipe.  Each 32-bit half is merged on its
+    // own: no carry can cross.
+    uint64_t c = mulwide(a0, b.m[0]) ^ mulwide(a1, b.m[3]) ^ mulwide(a2, b.m[2]) ^ mulwide(a3, b.m[1]);
+    uint32_t lo = (uint32_t)c & GIFT_M0, hi = (uint32_t)(c >> 32) & GIFT_M0;
+    c = mulwide(a0, b.m[1]) ^ mulwide(a1, b.m[0]) ^ mulwide(a2, b.m[3]) ^ mulwide(a3, b.m[2]);
+    lo = add_mul((uint32_t)c & GIFT_M1, lo);
+    hi = add_mul((uint32_t)(c >> 32) & GIFT_M1, hi);
+    c = mulwide(a0, b.m[2]) ^ mulwide(a1, b.m[1]) ^ mulwide(a2, b.m[0]) ^ mulwide(a3, b.m[3]);
+    lo = add_mul((uint32_t)c & GIFT_M2, lo);
+    hi = add_mul((uint32_t)(c >> 32) & GIFT_M2, hi);
+    c = mulwide(a0, b.m[3]) ^ mulwide(a1, b.m[2]) ^ mulwide(a2, b.m[1]) ^ mulwide(a3, b.m[0]);
+    lo = add_mul((uint32_t)c & GIFT_M3, lo);
+    hi = add_mul((uint32_t)(c >> 32) & GIFT_M3, hi);
+    return ((uint64_t)hi << 32) | lo;
 }
 
 // A fixed multiplier prepared for repeated use: the nine Karatsuba leaf
@@ -180,23 +222,45 @@ GIFT_HD void clmul128(const u128& a, const mulop& b, uint32_t r[8])
     r[7] = z2[3];
 }
 
-// Reduce a 256-bit polynomial modulo x^128 + x^7 + x^2 + x + 1.
+// Reduce a 256-bit polynomial modulo x^128 + x^7 + x^2 + x + 1: the high half h folds
+// down as h * (1 + x + x^2 + x^7).  Each shift of the 128-bit h by s bits is four
+// 32x32 -> 64 multiplies by 2^s (low word stays in place, high word carries into the next
+// word; the two never overlap, so they XOR straight into the sum).  The few bits pushed
+// past x^127 wrap around once more.
 GIFT_HD u128 reduce256(const uint32_t r[8])
 {
+#if !GIFT_REDUCE_ON_MUL
     const uint32_t h0 = r[4], h1 = r[5], h2 = r[6], h3 = r[7];
-    // t = h * (1 + x + x^2 + x^7), low 128 bits
     uint32_t t0 = h0 ^ (h0 << 1) ^ (h0 << 2) ^ (h0 << 7);
     uint32_t t1 = h1 ^ fshl(h0, h1, 1) ^ fshl(h0, h1, 2) ^ fshl(h0, h1, 7);
     uint32_t t2 = h2 ^ fshl(h1, h2, 1) ^ fshl(h1, h2, 2) ^ fshl(h1, h2, 7);
     uint32_t t3 = h3 ^ fshl(h2, h3, 1) ^ fshl(h2, h3, 2) ^ fshl(h2, h3, 7);
-    // the bits pushed past x^127 (at most 7 of them) wrap around once more
-    const uint32_t o = (h3 >> 31) ^ (h3 >> 30) ^ (h3 >> 25);
-    t0 ^= o ^ (o << 1) ^ (o << 2) ^ (o << 7);
+    const uint32_t ov = (h3 >> 31) ^ (h3 >> 30) ^ (h3 >> 25);
+    t0 ^= ov ^ (ov << 1) ^ (ov << 2) ^ (ov << 7);
+    u128 zz;
+    zz.w[0] = r[0] ^ t0; zz.w[1] = r[1] ^ t1; zz.w[2] = r[2] ^ t2; zz.w[3] = r[3] ^ t3;
+    return zz;
+#endif
+    const uint32_t k2 = GIFT_KMUL(1), k4 = GIFT_KMUL(2), k128 = GIFT_KMUL(3);
     u128 z;
-    z.w[0] = r[0] ^ t0;
-    z.w[1] = r[1] ^ t1;
-    z.w[2] = r[2] ^ t2;
-    z.w[3] = r[3] ^ t3;
+    // word 0 waits for the wrapped bits; words 1..3 take the carries of the word below
+    uint64_t a1 = mulwide(r[4], k2), a2 = mulwide(r[4], k4), a7 = mulwide(r[4], k128);
+    const uint32_t z0 = r[0] ^ r[4] ^ (uint32_t)a1 ^ (uint32_t)a2 ^ (uint32_t)a7;
+    uint32_t c1 = (uint32_t)(a1 >> 32), c2 = (uint32_t)(a2 >> 32), c7 = (uint32_t)(a7 >> 32);
+#if defined(__CUDA_ARCH__)
+#pragma unroll
+#endif
+    for (int k = 1; k < 4; k++) {
+        a1 = mulwide(r[4 + k], k2);
+        a2 = mulwide(r[4 + k], k4);
+        a7 = mulwide(r[4 + k], k128);
+        z.w[k] = r[k] ^ r[4 + k] ^ (uint32_t)a1 ^ (uint32_t)a2 ^ (uint32_t)a7 ^ c1 ^ c2 ^ c7;
+        c1 = (uint32_t)(a1 >> 32);
+        c2 = (uint32_t)(a2 >> 32);
+        c7 = (uint32_t)(a7 >> 32);
+    }
+    const uint32_t o = c1 ^ c2 ^ c7;                 // at most 7 bits past x^127
+    z.w[0] = z0 ^ o ^ (o * k2) ^ (o * k4) ^ (o * k128);
     return z;
 }
 

@@ -206,6 +206,102 @@ GIFT_HD u128 run_lane(const Tab& tb, const uint32_t* rk, const CtrPrefix& pre, c
     return sum;
 }
 
+// The same work as run_lane with one chain per lane, arranged for the hot loop:
+//  - rows of 32 blocks in which every lane has a full block run without predicates, the
+//    lane pointer advancing by 512 bytes per row; in paged mode this needs pages that are
+//    a multiple of 512 bytes, so that a row never straddles a page (otherwise the caller
+//    uses run_lane);
+//  - the loop is software pipelined: the keystream of row j and the hash update of row
+//    j-1 are independent, so the table lookups of the cipher and the multiplies and logic
+//    of the hash can interleave inside one warp;
+//  - the ragged last row (and a partial last block) goes through predicated code once.
+template <int MODE, class Tab>
+GIFT_HD u128 run_lane_rows(const Tab& tb, const uint32_t* rk, const CtrPrefix& pre, const mulop& hs,
+                           const u128* powtab, const uint8_t* src, uint8_t* dst, const SegAddr& addr,
+                           uint64_t seg_nblk, uint64_t run_first, uint32_t run_n, uint32_t tail, int lane)
+{
+    const bool has_partial = tail != 0 && run_first + run_n == seg_nblk;
+    const uint32_t n_full = run_n - (has_partial ? 1u : 0u);
+    const uint32_t rows = n_full >> 5;                      // rows in which all 32 lanes hold a full block
+    u128 acc = gf_zero();
+    uint32_t ctr = (uint32_t)(run_first + 2) + (uint32_t)lane;
+
+    // position of the run's first row
+    uint64_t pidx = 0, within = run_first * 16, base;
+    uint32_t rows_in_page = 0xFFFFFFFFu;                    // flat: never wraps
+    if (addr.table) {
+        pidx = within / addr.page_bytes;
+        within -= pidx * addr.page_bytes;
+        base = (uint64_t)(uint32_t)addr.table[addr.origin + pidx] * addr.page_bytes;
+        rows_in_page = (uint32_t)((addr.page_bytes - within) >> 9);
+    } else {
+        base = addr.origin;
+    }
+    uint64_t off = base + within + (uint64_t)lane * 16;     // this lane's block of the current row
+
+    Block c_prev;
+    c_prev.d[0] = c_prev.d[1] = c_prev.d[2] = c_prev.d[3] = 0;
+    bool pending = false;
+#pragma unroll 1
+    for (uint32_t j = 0; j < rows; j++) {
+        const Block d = load_block(src + off);
+        Block c = d;
+        if (MODE != MODE_VERIFY) {
+            uint32_t ks[4];
+            ctr_keystream(tb, rk, pre, ctr, ks);
+            Block o;
+            o.d[0] = d.d[0] ^ ks[0]; o.d[1] = d.d[1] ^ ks[1];
+            o.d[2] = d.d[2] ^ ks[2]; o.d[3] = d.d[3] ^ ks[3];
+            store_block(dst + off, o);
+            if (MODE == MODE_ENCRYPT) c = o;
+        }
+        // hash update of the previous row (the first pass multiplies zero, which stays zero)
+        acc = xor128(gfmul(acc, hs), block_to_field(c_prev.d[0], c_prev.d[1], c_prev.d[2], c_prev.d[3]));
+        c_prev = c;
+        pending = true;
+        ctr += 32;
+        off += 512;
+        if (--rows_in_page == 0) {                          // next page (uniform across the warp)
+            pidx++;
+            if (j + 1 < rows || (uint64_t)rows * 32 < run_n) {
+                base = (uint64_t)(uint32_t)addr.table[addr.origin + pidx] * addr.page_bytes;
+                off = base + (uint64_t)lane * 16;
+            }
+            rows_in_page = (uint32_t)(addr.page_bytes >> 9);
+        }
+    }
+    if (pending) acc = xor128(gfmul(acc, hs), block_to_field(c_prev.d[0], c_prev.d[1], c_prev.d[2], c_prev.d[3]));
+
+    // ragged last row: some lanes hold one more block, one of them possibly the partial block
+    const uint32_t i = rows * 32 + (uint32_t)lane;
+    uint32_t count = rows;                                  // blocks this lane has hashed
+    if (i < run_n) {
+        const bool partial = has_partial && i == run_n - 1;
+        const Block d = partial ? load_partial(src + off, tail) : load_block(src + off);
+        Block c = d;
+        if (MODE != MODE_VERIFY) {
+            uint32_t ks[4];
+            ctr_keystream(tb, rk, pre, ctr, ks);
+            Block o;
+            o.d[0] = d.d[0] ^ ks[0]; o.d[1] = d.d[1] ^ ks[1];
+            o.d[2] = d.d[2] ^ ks[2]; o.d[3] = d.d[3] ^ ks[3];
+            if (partial) {
+                store_partial(dst + off, o, tail);
+                mask_partial(o, tail);
+            } else {
+                store_block(dst + off, o);
+            }
+            if (MODE == MODE_ENCRYPT) c = o;
+        }
+        acc = xor128(gfmul(acc, hs), block_to_field(c.d[0], c.d[1], c.d[2], c.d[3]));
+        count++;
+    }
+    if (count == 0) return gf_zero();
+    const uint32_t i_last = (uint32_t)lane + (count - 1) * 32;
+    const uint64_t e = seg_nblk - run_first - i_last + 1;
+    return mul_by_power(acc, powtab, e);
+}
+
 // Tag from the combined hash S of all runs: T = (S + LEN*H) ^ E_K(J0), as four LE words.
 template <class Tab>
 GIFT_HD void finish_tag(const Tab& tb, const uint32_t* rk, const uint32_t h[4], const uint32_t nonce[3],

@@ -48,7 +48,7 @@ struct gift_ctx {
     uint32_t flags;
     int chains;                        // Horner chains per lane (1 or 2)
     int tables;                        // T-tables held in shared memory (2 or 4)
-    int threads;                       // threads per CTA of the cipher kernel (512 or 1024)
+    int threads;                       // threads per CTA of the cipher kernel (512, 768 or 1024)
     int num_sms;
     uint32_t* d_t0;                    // 256-entry T0 in global memory
     KeyHot* d_hot;                     // [max_users]
@@ -406,9 +406,15 @@ __global__ void __launch_bounds__(THREADS, 1) crypt_kernel(CallArgs a, const uin
         addr.page_bytes = a.page_bytes;
         addr.origin = a.page_table ? (uint64_t)seg.page0 : seg.offset;
 
-        const u128 part = run_lane<U, MODE>(tb, rk, pre, slot->hs[U - 1],
-                                            a.pow + (size_t)seg.owner * (POW_LEVELS * 256), a.src, a.dst, addr,
-                                            nblk, run_first, run_n, (uint32_t)(seg.len & 15), lane);
+        u128 part;
+        if (U == 1 && (a.page_table == nullptr || (a.page_bytes & 511) == 0)) {
+            // rows of 32 blocks never straddle a page: the pipelined row loop applies
+            part = run_lane_rows<MODE>(tb, rk, pre, slot->hs[0], a.pow + (size_t)seg.owner * (POW_LEVELS * 256),
+                                       a.src, a.dst, addr, nblk, run_first, run_n, (uint32_t)(seg.len & 15), lane);
+        } else {
+            part = run_lane<U, MODE>(tb, rk, pre, slot->hs[U - 1], a.pow + (size_t)seg.owner * (POW_LEVELS * 256),
+                                     a.src, a.dst, addr, nblk, run_first, run_n, (uint32_t)(seg.len & 15), lane);
+        }
         u128 sum;
         sum.w[0] = warp_xor(part.w[0]);
         sum.w[1] = warp_xor(part.w[1]);
@@ -682,6 +688,10 @@ int launch_crypt(gift_ctx* c, const CallArgs& a, cudaStream_t st)
         if (c->tables == 4) return launch_crypt_t<1, MODE, 4, 1024>(c, a, st);
         return launch_crypt_t<1, MODE, 2, 1024>(c, a, st);
     }
+    if (c->threads == 768) {
+        if (c->tables == 4) return launch_crypt_t<1, MODE, 4, 768>(c, a, st);
+        return launch_crypt_t<1, MODE, 2, 768>(c, a, st);
+    }
     if (c->tables == 4) {
         return c->chains == 2 ? launch_crypt_t<2, MODE, 4, 512>(c, a, st) : launch_crypt_t<1, MODE, 4, 512>(c, a, st);
     }
@@ -761,12 +771,12 @@ int gift_ctx_create(gift_ctx** out, int device, uint32_t max_users, uint32_t fla
 {
     if (!out || max_users == 0) return GIFT_E_INVAL;
     *out = nullptr;
-    int chains = (int)(flags & 0xFu), tables = (int)((flags >> 4) & 0xFu), threads = (int)((flags >> 8) & 0xFu) * 512;
+    int chains = (int)(flags & 0xFu), tables = (int)((flags >> 4) & 0xFu), threads = (int)((flags >> 8) & 0xFu) * 256;
     if (chains == 0) chains = 1;
     if (tables == 0) tables = 4;
-    if (threads == 0) threads = 512;
-    if ((chains != 1 && chains != 2) || (tables != 2 && tables != 4) || (threads != 512 && threads != 1024) ||
-        (threads == 1024 && chains != 1) || (flags >> 12))
+    if (threads == 0) threads = chains == 2 ? 512 : 768;
+    if ((chains != 1 && chains != 2) || (tables != 2 && tables != 4) || (threads != 512 && threads != 768 && threads != 1024) ||
+        (threads > 512 && chains != 1) || (flags >> 12))
         return GIFT_E_INVAL;
     if (max_users > (1u << 20)) return GIFT_E_RANGE;
     DeviceGuard g(device);

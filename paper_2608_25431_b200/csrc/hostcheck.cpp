@@ -120,14 +120,24 @@ static void seg_emulate(const uint8_t* key, const uint8_t* nonce12, const uint8_
         const uint32_t n = (uint32_t)(nblk - first < run_blocks ? nblk - first : run_blocks);
         for (int lane = 0; lane < 32; lane++) {
             u128 c;
-            if (mode == 0)
-                c = run_lane<U, MODE_ENCRYPT>(tab(), hot.rk, pre, hot.hs[U - 1], pow.data(), src, dst, addr,
+            if (U == 0) {                 // the row-wise, software-pipelined loop (chains == 0 selects it)
+                if (mode == 0)
+                    c = run_lane_rows<MODE_ENCRYPT>(tab(), hot.rk, pre, hot.hs[0], pow.data(), src, dst, addr,
+                                                    nblk, first, n, tail, lane);
+                else if (mode == 1)
+                    c = run_lane_rows<MODE_DECRYPT>(tab(), hot.rk, pre, hot.hs[0], pow.data(), src, dst, addr,
+                                                    nblk, first, n, tail, lane);
+                else
+                    c = run_lane_rows<MODE_VERIFY>(tab(), hot.rk, pre, hot.hs[0], pow.data(), src, dst, addr,
+                                                   nblk, first, n, tail, lane);
+            } else if (mode == 0)
+                c = run_lane<(U ? U : 1), MODE_ENCRYPT>(tab(), hot.rk, pre, hot.hs[U ? U - 1 : 0], pow.data(), src, dst, addr,
                                               nblk, first, n, tail, lane);
             else if (mode == 1)
-                c = run_lane<U, MODE_DECRYPT>(tab(), hot.rk, pre, hot.hs[U - 1], pow.data(), src, dst, addr,
+                c = run_lane<(U ? U : 1), MODE_DECRYPT>(tab(), hot.rk, pre, hot.hs[U ? U - 1 : 0], pow.data(), src, dst, addr,
                                               nblk, first, n, tail, lane);
             else
-                c = run_lane<U, MODE_VERIFY>(tab(), hot.rk, pre, hot.hs[U - 1], pow.data(), src, dst, addr,
+                c = run_lane<(U ? U : 1), MODE_VERIFY>(tab(), hot.rk, pre, hot.hs[U ? U - 1 : 0], pow.data(), src, dst, addr,
                                              nblk, first, n, tail, lane);
             s = xor128(s, c);
         }
@@ -145,7 +155,9 @@ void hc_segment(const uint8_t* key, const uint8_t* nonce12, const uint8_t* src, 
                 const int32_t* table, uint64_t page_bytes, uint64_t origin, uint64_t len,
                 uint32_t run_blocks, int chains, int mode, uint8_t* tag16)
 {
-    if (chains == 1)
+    if (chains == 0)
+        seg_emulate<0>(key, nonce12, src, dst, table, page_bytes, origin, len, run_blocks, mode, tag16);
+    else if (chains == 1)
         seg_emulate<1>(key, nonce12, src, dst, table, page_bytes, origin, len, run_blocks, mode, tag16);
     else
         seg_emulate<2>(key, nonce12, src, dst, table, page_bytes, origin, len, run_blocks, mode, tag16);

@@ -12,7 +12,7 @@ from gpu_harness import (dev, gpu_decrypt, gpu_encrypt, make_ctx, np_, oracle_de
 
 pytestmark = pytest.mark.gpu
 
-VARIANTS = [0, 0x21, 0x22, 0x41, 0x42, 0x241, 0x221]      # default, then (threads/512, tables, chains)
+VARIANTS = [0, 0x21, 0x22, 0x41, 0x42, 0x441, 0x421, 0x341, 0x241]      # default, then (threads/256, tables, chains)
 
 
 def _roundtrip_exact(w, flags=0, in_place=False):

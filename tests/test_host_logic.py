@@ -98,7 +98,7 @@ def test_power_table_matches_square_and_multiply(hc):
         assert o.tobytes() == power(e), e
 
 
-@pytest.mark.parametrize("chains", [1, 2])
+@pytest.mark.parametrize("chains", [0, 1, 2])
 def test_run_decomposition_reproduces_gcm(hc, chains):
     """Every (length, run length) split of a segment into runs, lanes and chains gives the oracle's bytes and tag."""
     rng = np.random.default_rng(3 + chains)
@@ -124,18 +124,20 @@ def test_run_decomposition_reproduces_gcm(hc, chains):
             assert tag3.tobytes() == ref_tag
 
 
-def test_paged_addressing_reproduces_gcm(hc):
+@pytest.mark.parametrize("pb,chains", [(160, 2), (160, 1), (512, 0), (1024, 0), (1536, 0)])
+def test_paged_addressing_reproduces_gcm(hc, pb, chains):
     rng = np.random.default_rng(9)
-    pb = 160
-    for n in [100, 160, 161, 1000, 3000, 3200]:
+    for n in [100, 160, 161, 1000, 3000, 3200, 5 * pb, 5 * pb + 1, 7 * pb - 1]:
         npg = (n + pb - 1) // pb
+        if npg + 3 > 40:
+            continue
         table = rng.permutation(40).astype(np.int32)
         buf = _u8(rng.bytes(40 * pb))
         out = buf.copy()
         tag = np.zeros(16, dtype=np.uint8)
         k, nonce = _u8(rng.bytes(16)), _u8(rng.bytes(12))
         hc.hc_segment(_p(k), _p(nonce), _p(buf), _p(out), _p(table), C.c_uint64(pb), C.c_uint64(3), C.c_uint64(n),
-                      C.c_uint32(64), 2, 0, _p(tag))
+                      C.c_uint32(64), chains, 0, _p(tag))
         sl = [(int(table[3 + i]) * pb, min(pb, n - i * pb)) for i in range(npg)]
         plain = b"".join(buf[o:o + l].tobytes() for o, l in sl)
         got = b"".join(out[o:o + l].tobytes() for o, l in sl)
