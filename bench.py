@@ -33,6 +33,11 @@ UNIT = "GB/s"
 # Integer work per 16-byte block of the best formulation known to this build (frozen; the
 # kernel's own instruction count is not used): T-table AES-CTR with the first round hoisted
 # and GHASH by masked integer multiplies with two Karatsuba levels.
+# DRAM bytes per payload byte of the cipher kernel, from the ncu capture summarised in
+# profiles/crypt_kernel_c3_2layers.md (dram__bytes_read.sum + dram__bytes_write.sum over the
+# payload of that launch); traffic grows in proportion to the payload.
+NCU_DRAM_BYTES_PER_PAYLOAD_BYTE = 1.926
+
 ALU_OPS_PER_BLOCK = 660          # logic / permute / shift / add lane-operations
 MUL_OPS_PER_BLOCK = 144          # 32x32 -> 64 multiplies
 LDS_OPS_PER_BLOCK = 150          # 4-byte shared-memory lookups
@@ -189,7 +194,7 @@ def main():
 
     import torch
     import torch.distributed as dist
-    from paper_2608_25431_b200 import binding, device_fill, workloads as W
+    from paper_2608_25431_b200 import binding, device_fill, replicas, workloads as W
 
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
@@ -260,12 +265,8 @@ def main():
     crypt_ms, crypt_n = ctx.timing_read()
     ctx.timing_enable(False)
     launches = ctx.launch_count() - l0 + (args.steps if flush is not None else 0) * 0
-    t = torch.tensor([total_ms], dtype=torch.float64, device="cuda")
-    if world > 1:
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-    total_ms_max = float(t.item())
+    value, total_ms_max = replicas.job_throughput(payload * args.steps, total_ms, "cuda")
     ms_per_step = total_ms_max / args.steps
-    value = world * payload / (ms_per_step * 1e-3) / 1e9
 
     # ---- roofline of the dominant kernel (the cipher kernel), bound by the integer pipes ----
     nblk = int(((w.segs["len"].astype(np.int64) + 15) // 16).sum())
@@ -286,7 +287,8 @@ def main():
     achieved_tops = ALU_OPS_PER_BLOCK * nblk / (kern_ms * 1e-3) / 1e12
     peak_tops = sms * r_alu * f / 1e12
     roofline = {"bound": "alu", "achieved": achieved_tops, "peak": peak_tops, "unit": "Top/s",
-                "frac": t_roof / (kern_ms * 1e-3), "traffic": None,
+                "frac": t_roof / (kern_ms * 1e-3), "traffic": NCU_DRAM_BYTES_PER_PAYLOAD_BYTE * payload,
+                "traffic_note": "bytes per launch: ncu DRAM bytes per payload byte on the 2-layer capture x this payload",
                 "kernel": "crypt_kernel", "kernel_ms": kern_ms, "kernel_launches": crypt_n,
                 "kernel_payload_gbs": payload / (kern_ms * 1e-3) / 1e9,
                 "hbm_achieved_gbs": 2.0 * payload / (kern_ms * 1e-3) / 1e9,
@@ -329,16 +331,31 @@ def main():
                          "identity_rule_us": rule_us}
 
     # ---- end to end from pinned host memory ----
+    # Every step uploads the whole plaintext pool from pinned host memory and downloads the
+    # ciphertext, tags and status words.  With a layer-major pool the work is cut into one
+    # chunk per layer over three streams (hostio.HostExporter) so that upload, cipher and
+    # download overlap; other workloads go through in one piece.
     if not args.no_e2e:
         try:
+            from paper_2608_25431_b200 import hostio
             h_in = torch.empty(w.buf_bytes, dtype=torch.uint8, pin_memory=True)
             h_out = torch.empty(w.buf_bytes, dtype=torch.uint8, pin_memory=True)
             h_tags = torch.empty((nseg, 16), dtype=torch.uint8, pin_memory=True)
             h_status = torch.empty(nseg, dtype=torch.int32, pin_memory=True)
             h_in.copy_(buf)
             k = max(1, min(args.steps, 5))
+            exporter = None
+            if args.workload == "c3":
+                n_slots = w.extra["n_slots"]
+                chunks = hostio.layer_chunks(w.extra["layers"], n_slots, n_slots * w.page_bytes)
+                exporter = hostio.HostExporter(w.max_users, w.user_ids, w.keys, local, 3, args.flags, n_slots)
 
             def e2e_step():
+                if exporter is not None:
+                    ctx.propagate_labels(binding.RULE_IDENTITY, [om_src], om, viol)
+                    exporter.export(h_in, h_out, buf, chunks, segs, tags, status, h_tags, h_status,
+                                    page_table=table, page_bytes=w.page_bytes, owner_map=om, unit_bytes=w.unit_bytes)
+                    return
                 buf.copy_(h_in, non_blocking=True)
                 ctx.propagate_labels(binding.RULE_IDENTITY, [om_src], om, viol)
                 ctx.seg_encrypt(buf, buf, segs, nseg, tags, status, page_table=table, page_bytes=w.page_bytes,
@@ -349,19 +366,21 @@ def main():
 
             e2e_step()
             barrier()
+            ok_e2e = not bool(h_status.any().item())
             a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
             a.record()
             for _ in range(k):
                 e2e_step()
             b.record()
             barrier()
-            t2 = torch.tensor([a.elapsed_time(b) / k], dtype=torch.float64, device="cuda")
-            if world > 1:
-                dist.all_reduce(t2, op=dist.ReduceOp.MAX)
-            e2e_ms = float(t2.item())
-            line["e2e"] = {"value": world * payload / e2e_ms / 1e6, "unit": UNIT,
+            e2e_value, e2e_ms = replicas.job_throughput(payload, a.elapsed_time(b) / k, "cuda")
+            line["e2e"] = {"value": e2e_value, "unit": UNIT,
                            "h2d_bytes_per_step": int(w.buf_bytes),
-                           "d2h_bytes_per_step": int(w.buf_bytes + nseg * 20), "steps": k, "ms_per_step": e2e_ms}
+                           "d2h_bytes_per_step": int(w.buf_bytes + nseg * 20), "steps": k, "ms_per_step": e2e_ms,
+                           "mode": "one chunk per layer on 3 streams" if exporter is not None else "one piece",
+                           "all_status_clear": ok_e2e}
+            if exporter is not None:
+                exporter.close()
             del h_in, h_out
         except RuntimeError as e:
             line["e2e"] = {"value": None, "unit": UNIT, "error": str(e)[:200]}

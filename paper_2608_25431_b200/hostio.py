@@ -1,0 +1,82 @@
+"""Export from pinned host memory, chunked so that copies overlap the cipher.
+
+A caller whose plaintext sits in pinned host memory (a swapped-out KV pool, paper sec. 4.5)
+needs host -> device copy, export, device -> host copy.  Done in one piece the three stages
+run back to back and PCIe idles while the cipher runs and the other way round.  Here the
+buffer is cut into chunks that no segment straddles (for the layer-major KV pool: one
+layer per chunk); chunk i uses stream i mod k, so the upload of one chunk, the cipher of
+the previous one and the download of the one before overlap.  Each stream has its own
+context, because a context's scratch belongs to one stream at a time.
+
+Only orchestration lives here: every byte is produced by gift_seg_encrypt.
+"""
+from __future__ import annotations
+
+from dataclasses import dataclass
+from typing import List, Optional
+
+import torch
+
+from . import binding
+
+
+@dataclass
+class Chunk:
+    byte_lo: int      # buffer range [byte_lo, byte_hi) that holds all bytes of the chunk's segments
+    byte_hi: int
+    seg_lo: int       # rows [seg_lo, seg_hi) of the segment table
+    seg_hi: int
+
+
+def layer_chunks(n_layers: int, segs_per_layer: int, bytes_per_layer: int) -> List[Chunk]:
+    """Chunks of a layer-major pool whose segment table is layer-major too."""
+    return [Chunk(l * bytes_per_layer, (l + 1) * bytes_per_layer, l * segs_per_layer, (l + 1) * segs_per_layer)
+            for l in range(n_layers)]
+
+
+class HostExporter:
+    """k contexts and streams that export chunks of a host buffer through one device buffer."""
+
+    def __init__(self, max_users: int, user_ids, keys, device: int = 0, n_streams: int = 3, flags: int = 0,
+                 max_segs_per_chunk: int = 1024):
+        self.ctxs = [binding.Ctx(max_users, device, flags) for _ in range(n_streams)]
+        for c in self.ctxs:
+            c.set_keys(user_ids, keys)
+            c.reserve(max_segs_per_chunk)
+        self.streams = [torch.cuda.Stream(device=device) for _ in range(n_streams)]
+
+    def close(self):
+        for c in self.ctxs:
+            c.close()
+
+    def launch_count(self) -> int:
+        return sum(c.launch_count() for c in self.ctxs)
+
+    def export(self, h_src: torch.Tensor, h_dst: torch.Tensor, d_buf: torch.Tensor, chunks: List[Chunk],
+               d_segs: torch.Tensor, d_tags: torch.Tensor, d_status: torch.Tensor, h_tags: torch.Tensor,
+               h_status: torch.Tensor, page_table: Optional[torch.Tensor] = None, page_bytes: int = 0,
+               owner_map: Optional[torch.Tensor] = None, unit_bytes: int = 0):
+        """Enqueue upload, export and download of every chunk; returns without waiting.
+
+        h_src, h_dst: pinned uint8 host tensors of the buffer's size; d_buf: device staging of
+        the same size; d_segs: the whole table on the device as uint8[nseg*40].
+        """
+        cur = torch.cuda.current_stream()
+        start = torch.cuda.Event()
+        start.record(cur)
+        for i, ch in enumerate(chunks):
+            st = self.streams[i % len(self.streams)]
+            ctx = self.ctxs[i % len(self.ctxs)]
+            st.wait_event(start)
+            with torch.cuda.stream(st):
+                d_buf[ch.byte_lo:ch.byte_hi].copy_(h_src[ch.byte_lo:ch.byte_hi], non_blocking=True)
+                n = ch.seg_hi - ch.seg_lo
+                ctx.seg_encrypt(d_buf, d_buf, d_segs[ch.seg_lo * 40: ch.seg_hi * 40], n,
+                                d_tags[ch.seg_lo:ch.seg_hi], d_status[ch.seg_lo:ch.seg_hi],
+                                page_table=page_table, page_bytes=page_bytes, owner_map=owner_map,
+                                unit_bytes=unit_bytes, stream=st.cuda_stream)
+                h_dst[ch.byte_lo:ch.byte_hi].copy_(d_buf[ch.byte_lo:ch.byte_hi], non_blocking=True)
+                h_tags[ch.seg_lo:ch.seg_hi].copy_(d_tags[ch.seg_lo:ch.seg_hi], non_blocking=True)
+                h_status[ch.seg_lo:ch.seg_hi].copy_(d_status[ch.seg_lo:ch.seg_hi], non_blocking=True)
+        for st in self.streams:
+            cur.wait_stream(st)
