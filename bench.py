@@ -38,6 +38,10 @@ UNIT = "GB/s"
 # payload of that launch); traffic grows in proportion to the payload.
 NCU_DRAM_BYTES_PER_PAYLOAD_BYTE = 1.926
 
+# ALU-pipe instructions per block the cipher kernel actually executes (ncu, same capture):
+# the tighter ceiling "if this very instruction stream issued at the pipe's full rate".
+EXECUTED_ALU_OPS_PER_BLOCK = 489
+
 ALU_OPS_PER_BLOCK = 660          # logic / permute / shift / add lane-operations
 MUL_OPS_PER_BLOCK = 144          # 32x32 -> 64 multiplies
 LDS_OPS_PER_BLOCK = 150          # 4-byte shared-memory lookups
@@ -296,6 +300,8 @@ def main():
                 "ceilings_gbs": {"alu": payload / t_alu / 1e9, "mul": payload / t_mul / 1e9,
                                  "lds": payload / t_lds / 1e9, "issue": payload / t_issue / 1e9,
                                  "hbm": payload / t_hbm / 1e9},
+                "frac_vs_executed_alu": (EXECUTED_ALU_OPS_PER_BLOCK * nblk / (sms * r_alu * f)) / (kern_ms * 1e-3),
+                "executed_alu_ops_per_block": EXECUTED_ALU_OPS_PER_BLOCK,
                 "sm_mhz_used": f_mhz,
                 "peak_source": "148 SMs x 64 integer lanes x sampled SM clock; HBM from MEASURED_PEAKS.json (of measured)"
                 if peaks else "fallback HBM 6650 GB/s (of fallback)"}
