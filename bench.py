@@ -331,7 +331,22 @@ def main():
                              ctx.seg_decrypt(buf, buf, segs, nseg, tags, status, page_table=table,
                                              page_bytes=w.page_bytes, owner_map=om, unit_bytes=w.unit_bytes)), n=3)
         rule_us = timed(lambda: ctx.propagate_labels(binding.RULE_IDENTITY, [om_src], om, viol), n=50) * 1e3
-        line["extra"] = {"verify_gbs": payload / ver / 1e6, "verify_all_ok": bool(ok_verify),
+        # token mode (one AES block per token, paper sec. 4.5): launch-latency bound
+        tok = {}
+        for nt in (256, 131328):
+            g = torch.Generator(device="cuda")
+            g.manual_seed(W.SEED_BASE + 50)
+            t_in = torch.randint(0, 32000, (nt,), generator=g, device="cuda", dtype=torch.int64)
+            n_in = torch.randint(0, 2**62, (nt,), generator=g, device="cuda", dtype=torch.int64)
+            own = torch.randint(0, len(w.user_ids), (nt,), generator=g, device="cuda", dtype=torch.int32)
+            c16 = torch.empty((nt, 16), dtype=torch.uint8, device="cuda")
+            stt = torch.empty(nt, dtype=torch.int32, device="cuda")
+            t_out = torch.empty(nt, dtype=torch.int64, device="cuda")
+            enc_ms = timed(lambda: ctx.tok_encrypt(t_in, n_in, own, 2, c16, stt), n=20)
+            dec_ms = timed(lambda: ctx.tok_decrypt(c16, own, 2, t_out, stt), n=20)
+            tok["%d_tokens" % nt] = {"encrypt_us": enc_ms * 1e3, "decrypt_us": dec_ms * 1e3,
+                                     "encrypt_mtok_s": nt / enc_ms / 1e3, "round_trip_ok": bool(torch.equal(t_out, t_in))}
+        line["extra"] = {"verify_gbs": payload / ver / 1e6, "verify_all_ok": bool(ok_verify), "token_mode": tok,
                          "encrypt_plus_decrypt_gbs": 2 * payload / dec / 1e6,
                          "decrypt_restores_ok": bool(not status.any().item()),
                          "identity_rule_us": rule_us}

@@ -185,6 +185,25 @@ int gift_verify_tags(gift_ctx* ctx, const void* src, uint64_t buf_bytes, const g
                      uint32_t nseg, const gift_pages* pages, const uint8_t* tags_in,
                      uint32_t* status, void* stream);
 
+/* Token mode (paper sec. 4.5, "Token encryption"): each token is encrypted on its own
+ * with a block cipher, not as part of a stream, because the framework splits and appends
+ * sequences; a 64-bit token is extended to 128 bits with a 64-bit nonce so that equal
+ * tokens give different ciphertexts, and the end-of-sequence token gets a special
+ * ciphertext that tells the framework that generation is complete.
+ * Here: block = LE64(token) || LE64(nonce), AES-128 under the key of owners[i]; a token
+ * equal to eos_token is replaced by the public marker of 16 bytes 0xFF.  tokens, nonces,
+ * owners (device arrays of n) give out16 (n x 16 bytes, 16-byte aligned) and status[i]
+ * (0, or GIFT_ST_NO_KEY with a zero block).  There is no integrity tag in this mode:
+ * decrypting under a wrong owner yields another token, never the plaintext. */
+int gift_tok_encrypt(gift_ctx* ctx, const uint64_t* tokens, const uint64_t* nonces, const int32_t* owners,
+                     uint32_t n, uint64_t eos_token, uint8_t* out16, uint32_t* status, void* stream);
+
+/* Inverse of gift_tok_encrypt with the CLAIMED owners (FIPS-197 inverse cipher): the nonce
+ * is dropped (nonces_out may be NULL), the marker decrypts to eos_token, a claimed owner
+ * without a key gives token 0 and GIFT_ST_NO_KEY. */
+int gift_tok_decrypt(gift_ctx* ctx, const uint8_t* in16, const int32_t* owners, uint32_t n, uint64_t eos_token,
+                     uint64_t* tokens_out, uint64_t* nonces_out, uint32_t* status, void* stream);
+
 /* A flow rule (paper sec. 4.3, "Generating IFT rules", steps 4 and 5): for
  * every output unit, its non-parameter sources must share one owner, which the
  * output receives; operands declared as parameters must be labelled PARAM.

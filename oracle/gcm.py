@@ -59,6 +59,14 @@ def aes128_encrypt_block(key, block) -> bytes:
     return out.tobytes()
 
 
+def aes128_decrypt_block(key, block) -> bytes:
+    k, b = _u8(key), _u8(block)
+    assert k.size == 16 and b.size == 16
+    out = np.zeros(16, dtype=np.uint8)
+    lib().gift_oracle_aes128_decrypt_block(_p(k), _p(b), _p(out))
+    return out.tobytes()
+
+
 def ctr32_xor(key, icb, data) -> bytes:
     k, i, d = _u8(key), _u8(icb), _u8(data)
     assert k.size == 16 and i.size == 16
@@ -177,6 +185,34 @@ def seg_decrypt(src, dst, segs, tags, user_ids, keys, max_users, page_table=None
     if rc != 0:
         raise ValueError("oracle seg_decrypt: bad call (%d)" % rc)
     return status[:n]
+
+
+def tok_encrypt(tokens, nonces, owners, eos_token, user_ids, keys, max_users):
+    """Token mode: (ciphertext uint8[n,16], status uint32[n])."""
+    t = np.ascontiguousarray(tokens, dtype=np.uint64)
+    nn = np.ascontiguousarray(nonces, dtype=np.uint64)
+    o = np.ascontiguousarray(owners, dtype=np.int32)
+    tab, has = _key_table(user_ids, keys, max_users)
+    n = t.size
+    out = np.zeros((max(n, 1), 16), dtype=np.uint8)
+    status = np.zeros(max(n, 1), dtype=np.uint32)
+    lib().gift_oracle_tok_encrypt(_p(t), _p(nn), _p(o), C.c_uint32(n), C.c_uint64(int(eos_token)), _p(tab), _p(has),
+                                  C.c_uint32(max_users), _p(out), _p(status))
+    return out[:n], status[:n]
+
+
+def tok_decrypt(ct, owners, eos_token, user_ids, keys, max_users):
+    """Token mode: (tokens uint64[n], nonces uint64[n], status uint32[n])."""
+    c = np.ascontiguousarray(ct, dtype=np.uint8).reshape(-1, 16)
+    o = np.ascontiguousarray(owners, dtype=np.int32)
+    tab, has = _key_table(user_ids, keys, max_users)
+    n = c.shape[0]
+    toks = np.zeros(max(n, 1), dtype=np.uint64)
+    nonces = np.zeros(max(n, 1), dtype=np.uint64)
+    status = np.zeros(max(n, 1), dtype=np.uint32)
+    lib().gift_oracle_tok_decrypt(_p(c), _p(o), C.c_uint32(n), C.c_uint64(int(eos_token)), _p(tab), _p(has),
+                                  C.c_uint32(max_users), _p(toks), _p(nonces), _p(status))
+    return toks[:n], nonces[:n], status[:n]
 
 
 def threads() -> int:

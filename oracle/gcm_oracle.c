@@ -152,6 +152,55 @@ void gift_oracle_aes128_encrypt_block(const uint8_t key[16], const uint8_t in[16
     aes128_cipher(rk, in, out);
 }
 
+/* InvCipher (FIPS-197 sec. 5.3): the rounds of Cipher undone in reverse order
+ * with InvShiftRows, InvSubBytes, AddRoundKey and InvMixColumns. */
+static uint8_t INV_SBOX[256];
+static int inv_sbox_ready = 0;
+
+static void aes128_inv_cipher(const uint8_t rk[176], const uint8_t in[16], uint8_t out[16])
+{
+    if (!inv_sbox_ready) {
+        for (int x = 0; x < 256; x++) INV_SBOX[SBOX[x]] = (uint8_t)x;
+        inv_sbox_ready = 1;
+    }
+    uint8_t s[4][4];
+    for (int c = 0; c < 4; c++)
+        for (int r = 0; r < 4; r++) s[r][c] = in[r + 4 * c] ^ rk[160 + r + 4 * c];
+    for (int round = 9; round >= 0; round--) {
+        /* InvShiftRows: row r rotates right by r */
+        for (int r = 1; r < 4; r++) {
+            uint8_t row[4];
+            for (int c = 0; c < 4; c++) row[(c + r) & 3] = s[r][c];
+            for (int c = 0; c < 4; c++) s[r][c] = row[c];
+        }
+        /* InvSubBytes */
+        for (int r = 0; r < 4; r++)
+            for (int c = 0; c < 4; c++) s[r][c] = INV_SBOX[s[r][c]];
+        /* AddRoundKey */
+        for (int c = 0; c < 4; c++)
+            for (int r = 0; r < 4; r++) s[r][c] ^= rk[16 * round + r + 4 * c];
+        /* InvMixColumns: circulant (0e 0b 0d 09), skipped after the last AddRoundKey */
+        if (round != 0) {
+            for (int c = 0; c < 4; c++) {
+                uint8_t a0 = s[0][c], a1 = s[1][c], a2 = s[2][c], a3 = s[3][c];
+                s[0][c] = gf256_mul(a0, 0x0e) ^ gf256_mul(a1, 0x0b) ^ gf256_mul(a2, 0x0d) ^ gf256_mul(a3, 0x09);
+                s[1][c] = gf256_mul(a0, 0x09) ^ gf256_mul(a1, 0x0e) ^ gf256_mul(a2, 0x0b) ^ gf256_mul(a3, 0x0d);
+                s[2][c] = gf256_mul(a0, 0x0d) ^ gf256_mul(a1, 0x09) ^ gf256_mul(a2, 0x0e) ^ gf256_mul(a3, 0x0b);
+                s[3][c] = gf256_mul(a0, 0x0b) ^ gf256_mul(a1, 0x0d) ^ gf256_mul(a2, 0x09) ^ gf256_mul(a3, 0x0e);
+            }
+        }
+    }
+    for (int c = 0; c < 4; c++)
+        for (int r = 0; r < 4; r++) out[r + 4 * c] = s[r][c];
+}
+
+void gift_oracle_aes128_decrypt_block(const uint8_t key[16], const uint8_t in[16], uint8_t out[16])
+{
+    uint8_t rk[176];
+    gift_oracle_aes128_key_expand(key, rk);
+    aes128_inv_cipher(rk, in, out);
+}
+
 /* ------------------------------------------------------------------------ */
 /* CTR (SP 800-38A sec. 6.5) with the 32-bit increment of SP 800-38D sec. 6.2 */
 /* ------------------------------------------------------------------------ */
@@ -518,3 +567,69 @@ int gift_oracle_seg_decrypt(const uint8_t* src, uint8_t* dst, uint64_t buf_bytes
     }
     return failed ? -2 : 0;
 }
+
+/* ------------------------------------------------------------------------ */
+/* Token mode (paper sec. 4.5, "Token encryption")                            */
+/* ------------------------------------------------------------------------ */
+
+/* Each 64-bit token is extended to 128 bits with a 64-bit nonce and passed
+ * through the block cipher under its owner's key, so that equal tokens do not
+ * give equal ciphertexts and the framework can still split and append
+ * sequences token by token.  Layout taken here: bytes 0-7 the token, bytes
+ * 8-15 the nonce, both little-endian.  The end-of-sequence token gets a fixed
+ * public marker instead of a ciphertext (16 bytes 0xFF) so that the framework
+ * can see that generation has ended.  Decryption applies the inverse cipher
+ * and drops the nonce; the marker decrypts to the end-of-sequence token.
+ * Status: ST_NO_KEY when the owner has no key (output zero). */
+static void put_le64(uint8_t* p, uint64_t v)
+{
+    for (int i = 0; i < 8; i++) p[i] = (uint8_t)(v >> (8 * i));
+}
+
+static uint64_t get_le64(const uint8_t* p)
+{
+    uint64_t v = 0;
+    for (int i = 7; i >= 0; i--) v = (v << 8) | p[i];
+    return v;
+}
+
+void gift_oracle_tok_encrypt(const uint64_t* tokens, const uint64_t* nonces, const int32_t* owners,
+                             uint32_t n, uint64_t eos_token, const uint8_t* keys,
+                             const uint8_t* has_key, uint32_t max_users, uint8_t* out16, uint32_t* status)
+{
+    gift_oracle_init();
+    for (uint32_t i = 0; i < n; i++) {
+        uint8_t* o = out16 + 16 * (uint64_t)i;
+        int ok = owners[i] >= 0 && (uint32_t)owners[i] < max_users && has_key[owners[i]];
+        status[i] = ok ? 0 : ST_NO_KEY;
+        if (!ok) { memset(o, 0, 16); continue; }
+        if (tokens[i] == eos_token) { memset(o, 0xFF, 16); continue; }
+        uint8_t blk[16];
+        put_le64(blk, tokens[i]);
+        put_le64(blk + 8, nonces[i]);
+        gift_oracle_aes128_encrypt_block(keys + 16 * (uint64_t)owners[i], blk, o);
+    }
+}
+
+void gift_oracle_tok_decrypt(const uint8_t* in16, const int32_t* owners, uint32_t n, uint64_t eos_token,
+                             const uint8_t* keys, const uint8_t* has_key, uint32_t max_users,
+                             uint64_t* tokens_out, uint64_t* nonces_out, uint32_t* status)
+{
+    gift_oracle_init();
+    for (uint32_t i = 0; i < n; i++) {
+        const uint8_t* c = in16 + 16 * (uint64_t)i;
+        int ok = owners[i] >= 0 && (uint32_t)owners[i] < max_users && has_key[owners[i]];
+        status[i] = ok ? 0 : ST_NO_KEY;
+        tokens_out[i] = 0;
+        if (nonces_out) nonces_out[i] = 0;
+        if (!ok) continue;
+        int marker = 1;
+        for (int k = 0; k < 16; k++) marker &= c[k] == 0xFF;
+        if (marker) { tokens_out[i] = eos_token; continue; }
+        uint8_t blk[16];
+        gift_oracle_aes128_decrypt_block(keys + 16 * (uint64_t)owners[i], c, blk);
+        tokens_out[i] = get_le64(blk);
+        if (nonces_out) nonces_out[i] = get_le64(blk + 8);
+    }
+}
+

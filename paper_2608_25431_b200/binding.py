@@ -24,7 +24,7 @@ STATIC_MAX_SEGS = 65536
 EXPORTS = [
     "gift_ctx_create", "gift_ctx_destroy", "gift_ctx_reserve", "gift_set_keys", "gift_clear_keys",
     "gift_seg_encrypt", "gift_seg_encrypt_static", "gift_seg_decrypt", "gift_verify_tags",
-    "gift_propagate_labels",
+    "gift_propagate_labels", "gift_tok_encrypt", "gift_tok_decrypt",
     "gift_strerror", "gift_version", "gift_launch_count", "gift_timing_enable", "gift_timing_read",
     "gift_probe_pipe",
 ]
@@ -75,6 +75,10 @@ def lib():
                                        C.POINTER(_Pages), C.c_void_p, C.c_void_p, C.c_void_p]
         l.gift_propagate_labels.argtypes = [C.c_void_p, C.POINTER(_Rule), C.POINTER(C.c_void_p), C.c_void_p,
                                             C.c_void_p, C.c_void_p]
+        l.gift_tok_encrypt.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_uint32, C.c_uint64,
+                                       C.c_void_p, C.c_void_p, C.c_void_p]
+        l.gift_tok_decrypt.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_uint32, C.c_uint64, C.c_void_p,
+                                       C.c_void_p, C.c_void_p, C.c_void_p]
         l.gift_strerror.restype = C.c_char_p
         l.gift_strerror.argtypes = [C.c_int]
         l.gift_version.restype = C.c_uint32
@@ -216,6 +220,16 @@ class Ctx:
         arr = (C.c_void_p * len(in_maps))(*[m.data_ptr() for m in in_maps])
         _check(lib().gift_propagate_labels(self._h, C.byref(rule), arr, _dev(out_map), _dev(viol),
                                            _stream_ptr(stream)), "gift_propagate_labels")
+
+    def tok_encrypt(self, tokens, nonces, owners, eos_token, out16, status, stream=None):
+        _check(lib().gift_tok_encrypt(self._h, _dev(tokens), _dev(nonces), _dev(owners), tokens.numel(),
+                                      int(eos_token), _dev(out16), _dev(status), _stream_ptr(stream)),
+               "gift_tok_encrypt")
+
+    def tok_decrypt(self, in16, owners, eos_token, tokens_out, status, nonces_out=None, stream=None):
+        _check(lib().gift_tok_decrypt(self._h, _dev(in16), _dev(owners), owners.numel(), int(eos_token),
+                                      _dev(tokens_out), _dev(nonces_out), _dev(status), _stream_ptr(stream)),
+               "gift_tok_decrypt")
 
     def launch_count(self) -> int:
         return int(lib().gift_launch_count(self._h))

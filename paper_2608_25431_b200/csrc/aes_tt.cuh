@@ -160,6 +160,50 @@ GIFT_HD void aes128_encrypt(const Tab& tb, const uint32_t* rk, uint32_t s[4])
     aes_last_round(tb, s, rk + 40);
 }
 
+// ---- inverse cipher (FIPS-197 sec. 5.3), used only by the token mode ----
+//
+// Written out plainly: InvShiftRows + InvSubBytes through a 256-byte inverse S-box,
+// AddRoundKey, and InvMixColumns computed on four packed bytes at a time.  Token batches
+// are small (the kernel is bound by launch latency), so no tables are built for it.
+
+// multiply each of the four packed bytes by x in GF(2^8)
+GIFT_HD uint32_t xtime4(uint32_t w)
+{
+    return ((w & 0x7F7F7F7Fu) << 1) ^ (((w >> 7) & 0x01010101u) * 0x1Bu);
+}
+
+GIFT_HD uint32_t rotr32(uint32_t x, int s)
+{
+    return (x >> s) | (x << (32 - s));
+}
+
+// One column: out row r = 0e*a_r ^ 0b*a_(r+1) ^ 0d*a_(r+2) ^ 09*a_(r+3)
+GIFT_HD uint32_t inv_mix_column(uint32_t w)
+{
+    const uint32_t w2 = xtime4(w), w4 = xtime4(w2), w8 = xtime4(w4);
+    const uint32_t w9 = w8 ^ w, wb = w9 ^ w2, wd = w9 ^ w4, we = w8 ^ w4 ^ w2;
+    return we ^ rotr32(wb, 8) ^ rotr32(wd, 16) ^ rotr32(w9, 24);
+}
+
+GIFT_HD void aes128_decrypt(const uint8_t* isbox, const uint32_t* rk, uint32_t s[4])
+{
+    s[0] ^= rk[40]; s[1] ^= rk[41]; s[2] ^= rk[42]; s[3] ^= rk[43];
+    for (int round = 9; round >= 0; round--) {
+        uint32_t t[4];
+        // InvShiftRows then InvSubBytes: output column c, row r comes from column (c - r) mod 4
+        for (int c = 0; c < 4; c++) {
+            t[c] = (uint32_t)isbox[s[c] & 0xFFu] |
+                   ((uint32_t)isbox[(s[(c + 3) & 3] >> 8) & 0xFFu] << 8) |
+                   ((uint32_t)isbox[(s[(c + 2) & 3] >> 16) & 0xFFu] << 16) |
+                   ((uint32_t)isbox[(s[(c + 1) & 3] >> 24) & 0xFFu] << 24);
+        }
+        for (int c = 0; c < 4; c++) {
+            const uint32_t v = t[c] ^ rk[4 * round + c];
+            s[c] = round != 0 ? inv_mix_column(v) : v;
+        }
+    }
+}
+
 // ---- CTR with GCM's counter layout (SP 800-38D sec. 7.1) ----
 //
 // Counter block = nonce (12 bytes) || BE32(ctr).  Only the last column varies

@@ -73,7 +73,7 @@ GIFT_HD uint64_t mulwide(uint32_t a, uint32_t b)
 // not a compile-time constant; constant memory that the host could rewrite is opaque
 // enough.  The values never change.
 #if defined(__CUDACC__)
-__constant__ uint32_t gift_kmul[4] = {1u, 2u, 4u, 128u};
+static __constant__ uint32_t gift_kmul[4] = {1u, 2u, 4u, 128u};
 #endif
 static const uint32_t gift_kmul_host[4] = {1u, 2u, 4u, 128u};
 #if defined(__CUDA_ARCH__)

@@ -30,55 +30,7 @@ using namespace gift;
 
 #define GIFT_VERSION 100u   // 0.1.0
 
-// ---------------------------------------------------------------------------
-// context
-// ---------------------------------------------------------------------------
-
-struct Globals {
-    unsigned long long total_blocks;   // 16-byte blocks of all accepted segments
-    uint32_t total_runs;
-    uint32_t run_blocks;               // blocks per run chosen for this call
-    uint32_t work;                     // next run to hand out
-    uint32_t pad[3];
-};
-
-struct gift_ctx {
-    int device;
-    uint32_t max_users;
-    uint32_t flags;
-    int chains;                        // Horner chains per lane (1 or 2)
-    int tables;                        // T-tables held in shared memory (2 or 4)
-    int threads;                       // threads per CTA of the cipher kernel (512, 768 or 1024)
-    int num_sms;
-    uint32_t* d_t0;                    // 256-entry T0 in global memory
-    KeyHot* d_hot;                     // [max_users]
-    u128* d_pow;                       // [max_users][POW_LEVELS*256]
-    uint8_t* h_stage;                  // pinned staging for keys
-    uint32_t stage_cap;                // users the staging buffers hold
-    int32_t* d_stage_ids;
-    uint8_t* d_stage_keys;
-    uint32_t seg_cap;
-    uint32_t* d_run_prefix;            // [seg_cap + 1]
-    uint4* d_acc;                      // [seg_cap]
-    uint32_t* d_ticket;                // [seg_cap]
-    Globals* d_glob;
-    int32_t* d_snapshot;               // label snapshot for aliased rules
-    uint32_t snapshot_cap;
-    uint64_t launches;
-    int timing;                        // record events around the cipher kernel
-    uint32_t n_timed;
-    cudaEvent_t* ev;                   // 2 * MAX_TIMED events, created on first enable
-};
-
-#define MAX_TIMED 1024u
-
-#define CU_TRY(expr)                                   \
-    do {                                               \
-        cudaError_t e_ = (expr);                       \
-        if (e_ != cudaSuccess) {                       \
-            return e_ == cudaErrorMemoryAllocation ? GIFT_E_NOMEM : GIFT_E_CUDA; \
-        }                                              \
-    } while (0)
+#include "gift_internal.cuh"
 
 namespace {
 
@@ -86,9 +38,10 @@ namespace {
 // tables and keys
 // ---------------------------------------------------------------------------
 
-__global__ void init_t0_kernel(uint32_t* t0)
+__global__ void init_t0_kernel(uint32_t* t0, uint8_t* isbox)
 {
     t0[threadIdx.x] = t0_entry(threadIdx.x);
+    isbox[sbox_entry(threadIdx.x)] = (uint8_t)threadIdx.x;      // the S-box is a permutation
 }
 
 // Four threads per user: each derives the key schedule and H, thread m builds
@@ -626,20 +579,6 @@ __global__ void viol_init_kernel(uint32_t* viol)
 // host side
 // ---------------------------------------------------------------------------
 
-struct DeviceGuard {
-    int prev;
-    bool ok;
-    explicit DeviceGuard(int dev) : prev(-1), ok(false)
-    {
-        if (cudaGetDevice(&prev) != cudaSuccess) return;
-        ok = prev == dev || cudaSetDevice(dev) == cudaSuccess;
-    }
-    ~DeviceGuard()
-    {
-        if (ok && prev >= 0) cudaSetDevice(prev);
-    }
-};
-
 int ensure_scratch(gift_ctx* c, uint32_t nseg)
 {
     if (nseg <= c->seg_cap) return GIFT_OK;
@@ -796,13 +735,14 @@ int gift_ctx_create(gift_ctx** out, int device, uint32_t max_users, uint32_t fla
     c->num_sms = prop.multiProcessorCount;
     auto fail = [&](int code) { gift_ctx_destroy(c); return code; };
     if (cudaMalloc(&c->d_t0, 256 * sizeof(uint32_t)) != cudaSuccess) return fail(GIFT_E_NOMEM);
+    if (cudaMalloc(&c->d_isbox, 256) != cudaSuccess) return fail(GIFT_E_NOMEM);
     if (cudaMalloc(&c->d_hot, (size_t)max_users * sizeof(KeyHot)) != cudaSuccess) return fail(GIFT_E_NOMEM);
     if (cudaMalloc(&c->d_pow, (size_t)max_users * POW_LEVELS * 256 * sizeof(u128)) != cudaSuccess) return fail(GIFT_E_NOMEM);
     if (cudaMalloc(&c->d_glob, sizeof(Globals)) != cudaSuccess) return fail(GIFT_E_NOMEM);
     if (cudaMemset(c->d_hot, 0, (size_t)max_users * sizeof(KeyHot)) != cudaSuccess) return fail(GIFT_E_CUDA);
     if (cudaMemset(c->d_pow, 0, (size_t)max_users * POW_LEVELS * 256 * sizeof(u128)) != cudaSuccess) return fail(GIFT_E_CUDA);
     if (cudaMemset(c->d_glob, 0, sizeof(Globals)) != cudaSuccess) return fail(GIFT_E_CUDA);
-    init_t0_kernel<<<1, 256>>>(c->d_t0);
+    init_t0_kernel<<<1, 256>>>(c->d_t0, c->d_isbox);
     c->launches++;
     if (cudaDeviceSynchronize() != cudaSuccess) return fail(GIFT_E_CUDA);
     rc = ensure_scratch(c, 1024);
@@ -821,7 +761,7 @@ int gift_ctx_destroy(gift_ctx* c)
         if (c->d_pow) cudaMemset(c->d_pow, 0, (size_t)c->max_users * POW_LEVELS * 256 * sizeof(u128));
         if (c->d_stage_keys) cudaMemset(c->d_stage_keys, 0, (size_t)c->stage_cap * 16);
         cudaDeviceSynchronize();
-        cudaFree(c->d_t0); cudaFree(c->d_hot); cudaFree(c->d_pow); cudaFree(c->d_glob);
+        cudaFree(c->d_t0); cudaFree(c->d_isbox); cudaFree(c->d_hot); cudaFree(c->d_pow); cudaFree(c->d_glob);
         cudaFree(c->d_run_prefix); cudaFree(c->d_acc); cudaFree(c->d_ticket);
         cudaFree(c->d_stage_ids); cudaFree(c->d_stage_keys); cudaFree(c->d_snapshot);
         if (c->h_stage) {

@@ -75,6 +75,18 @@ void hc_aes_encrypt(const uint8_t* key, const uint8_t* in, uint8_t* out)
     store_block(out, b);
 }
 
+void hc_aes_decrypt(const uint8_t* key, const uint8_t* in, uint8_t* out)
+{
+    uint32_t k[4], rk[44];
+    key_words(key, k);
+    aes128_expand_key(tab(), k, rk);
+    uint8_t isbox[256];
+    for (uint32_t x = 0; x < 256; x++) isbox[sbox_entry(x)] = (uint8_t)x;
+    Block b = load_block(in);
+    aes128_decrypt(isbox, rk, b.d);
+    store_block(out, b);
+}
+
 // H^e through the 4-level power table, as block bytes.
 void hc_power(const uint8_t* key, uint64_t e, uint8_t* out)
 {

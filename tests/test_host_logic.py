@@ -78,6 +78,15 @@ def test_table_cipher_and_key_schedule_match_oracle(hc):
         assert rk.tobytes() == gcm.key_expand(k).tobytes()
 
 
+def test_inverse_cipher_matches_oracle(hc):
+    rng = np.random.default_rng(5)
+    for _ in range(300):
+        k, b = _u8(rng.bytes(16)), _u8(rng.bytes(16))
+        o = np.zeros(16, dtype=np.uint8)
+        hc.hc_aes_decrypt(_p(k), _p(b), _p(o))
+        assert o.tobytes() == gcm.aes128_decrypt_block(k, b)
+
+
 def test_power_table_matches_square_and_multiply(hc):
     rng = np.random.default_rng(2)
     k = _u8(rng.bytes(16))

@@ -263,3 +263,43 @@ def test_ghash_zero_padding_and_aad_layout():
     for blk in (a + bytes(11), c[:16], c[16:] + bytes(11), lenblk):
         y = gcm.gf128_mul(_xor(y, blk), h)
     assert gcm.ghash(h, a, c) == y
+
+
+# ---- inverse cipher and token mode ------------------------------------------------
+
+def test_inverse_cipher_vs_openssl_and_published_example():
+    rng = np.random.default_rng(10)
+    for row in _kat("block"):
+        _, key, pt, ct = row
+        assert gcm.aes128_decrypt_block(_hex(key), _hex(ct)) == _hex(pt)      # FIPS-197 App. C.1 inverse cipher
+    for _ in range(500):
+        k, b = rng.bytes(16), rng.bytes(16)
+        dec = Cipher(algorithms.AES(k), modes.ECB()).decryptor().update(b)
+        assert gcm.aes128_decrypt_block(k, b) == dec
+        assert gcm.aes128_decrypt_block(k, gcm.aes128_encrypt_block(k, b)) == b
+
+
+def test_token_mode_layout_marker_and_round_trip():
+    rng = np.random.default_rng(11)
+    ids = np.arange(4, dtype=np.int32)
+    keys = np.frombuffer(rng.bytes(64), dtype=np.uint8).reshape(4, 16)
+    eos = 2
+    toks = np.array([17, 2, 17, 31999, 2**63 + 5, 17], dtype=np.uint64)
+    nonces = rng.integers(0, 2**63, size=6, dtype=np.uint64)
+    owners = np.array([0, 1, 0, 3, 2, 9], dtype=np.int32)          # user 9 has no key
+    ct, st = gcm.tok_encrypt(toks, nonces, owners, eos, ids, keys, 16)
+    assert st.tolist() == [0, 0, 0, 0, 0, 8] and not ct[5].any()
+    assert (ct[1] == 0xFF).all()                                   # the end-of-sequence marker
+    # one cipher block per token: bytes 0-7 token, 8-15 nonce, little-endian, under the owner's key
+    blk = int(toks[0]).to_bytes(8, "little") + int(nonces[0]).to_bytes(8, "little")
+    assert ct[0].tobytes() == _ecb(keys[0].tobytes(), blk)
+    assert ct[0].tobytes() != ct[2].tobytes()                      # same token, same key, other nonce
+    t2, n2, st2 = gcm.tok_decrypt(ct, owners, eos, ids, keys, 16)
+    assert st2.tolist() == [0, 0, 0, 0, 0, 8]
+    assert t2[:5].tolist() == toks[:5].tolist() and t2[5] == 0
+    assert n2[[0, 2, 3, 4]].tolist() == nonces[[0, 2, 3, 4]].tolist()
+    # a wrong claimed owner yields another token, never the plaintext (paper sec. 3, step 3)
+    wrong = owners.copy()
+    wrong[0] = 1
+    t3, _, _ = gcm.tok_decrypt(ct, wrong, eos, ids, keys, 16)
+    assert t3[0] != toks[0]
