@@ -66,16 +66,16 @@ GIFT_HD uint64_t mulwide(uint32_t a, uint32_t b)
     return (uint64_t)a * (uint64_t)b;
 }
 
-// Small multipliers (1, 2, 4, 128) that the compiler cannot see through.  On this GPU
+// Small multipliers (1, 2, 4, 128, 256) that the compiler cannot see through.  On this GPU
 // logic, permute and shift instructions share one pipe, which binds the cipher kernel,
 // while the multiply pipe is mostly idle.  An add written as a*1 + b, or a shift written
 // as a 32x32 -> 64 multiply by 2^s, stays a multiply instruction only if the factor is
 // not a compile-time constant; constant memory that the host could rewrite is opaque
 // enough.  The values never change.
 #if defined(__CUDACC__)
-static __constant__ uint32_t gift_kmul[4] = {1u, 2u, 4u, 128u};
+static __constant__ uint32_t gift_kmul[5] = {1u, 2u, 4u, 128u, 256u};
 #endif
-static const uint32_t gift_kmul_host[4] = {1u, 2u, 4u, 128u};
+static const uint32_t gift_kmul_host[5] = {1u, 2u, 4u, 128u, 256u};
 #if defined(__CUDA_ARCH__)
 #define GIFT_KMUL(i) gift_kmul[i]
 #else

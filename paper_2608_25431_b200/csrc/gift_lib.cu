@@ -268,17 +268,34 @@ extern __shared__ __align__(16) unsigned char smem_raw[];
 // byte 1 of the offset, so one byte-permute builds the address and the bank is
 // always the lane's own.  With NT == 2 only T0 and T1 are stored; T2 and T3 are
 // their 16-bit rotations.
+#ifndef GIFT_K3_ON_MUL
+#define GIFT_K3_ON_MUL 0   // measured: the two extra issue slots cost more than the freed logic slot (406 vs 421 GB/s)
+#endif
+
 template <int NT>
 struct SmemTab {
     uint32_t lb0, lb1;     // lane*4 and lane*4 + 128
+    // byte offset of entry (byte K of w) for this lane: index in byte 1, lane offset in byte 0
+    template <int K>
+    __device__ __forceinline__ uint32_t offset(uint32_t w, uint32_t lb) const
+    {
+#if GIFT_K3_ON_MUL
+        if (K == 3) {
+            // the top byte through the multiply pipe: (w * 256) >> 32 = w >> 24, then * 256 + lane offset
+            const uint32_t k256 = GIFT_KMUL(4);
+            const uint32_t top = (uint32_t)(((uint64_t)w * k256) >> 32);
+            return top * k256 + lb;
+        }
+#endif
+        return __byte_perm(w, lb, 0x7604u | (K << 4));
+    }
     template <int T, int K>
     __device__ __forceinline__ uint32_t look(uint32_t w) const
     {
+        const uint32_t off = offset<K>(w, (T & 1) ? lb1 : lb0);
         if (NT == 4) {
-            const uint32_t off = __byte_perm(w, (T & 1) ? lb1 : lb0, 0x7604u | (K << 4));
             return *reinterpret_cast<const uint32_t*>(smem_raw + (T >> 1) * 65536 + off);
         } else {
-            const uint32_t off = __byte_perm(w, (T & 1) ? lb1 : lb0, 0x7604u | (K << 4));
             const uint32_t v = *reinterpret_cast<const uint32_t*>(smem_raw + off);
             return (T >> 1) ? __byte_perm(v, 0u, 0x1032u) : v;
         }
@@ -286,8 +303,7 @@ struct SmemTab {
     template <int K>
     __device__ __forceinline__ uint32_t sub(uint32_t w) const
     {
-        const uint32_t off = __byte_perm(w, lb0, 0x7604u | (K << 4));
-        return *reinterpret_cast<const uint32_t*>(smem_raw + off);
+        return *reinterpret_cast<const uint32_t*>(smem_raw + offset<K>(w, lb0));
     }
 };
 

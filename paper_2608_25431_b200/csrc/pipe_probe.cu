@@ -86,6 +86,11 @@ __global__ void __launch_bounds__(1024, 1) probe_kernel(uint32_t iters, uint32_t
                 } else if (KIND == 17) {  // logic + permute (both integer pipe)
                     asm volatile("lop3.b32 %0, %0, %1, %2, 0x96;" : "+r"(x[c]) : "r"(k1), "r"(k2));
                     asm volatile("prmt.b32 %0, %0, %1, 0x2103;" : "+r"(x[c]) : "r"(k1));
+                } else if (KIND == 18) {  // high half of a 32x32 multiply
+                    asm volatile("mul.hi.u32 %0, %0, %1;" : "+r"(x[c]) : "r"(k1));
+                } else if (KIND == 19) {  // logic + high-half multiply
+                    asm volatile("lop3.b32 %0, %0, %1, %2, 0x96;" : "+r"(x[c]) : "r"(k1), "r"(k2));
+                    asm volatile("mul.hi.u32 %0, %1, %2;" : "=r"(*reinterpret_cast<uint32_t*>(&w[c])) : "r"(k2), "r"(k1));
                 } else if (KIND == 8) {   // logic and shared-memory loads interleaved
                     asm volatile("lop3.b32 %0, %0, %1, %2, 0x96;" : "+r"(x[c]) : "r"(k1), "r"(k2));
                     w[c] = vtab[lane4 + (c << 5)];
@@ -154,6 +159,8 @@ extern "C" int gift_probe_pipe(int device, int kind, uint32_t iters, double* lan
     case 15: e = run_probe<15>(sms, iters, d_cycles, d_sink, &ms); break;
     case 16: e = run_probe<16>(sms, iters, d_cycles, d_sink, &ms); break;
     case 17: e = run_probe<17>(sms, iters, d_cycles, d_sink, &ms); break;
+    case 18: e = run_probe<18>(sms, iters, d_cycles, d_sink, &ms); break;
+    case 19: e = run_probe<19>(sms, iters, d_cycles, d_sink, &ms); break;
     default: cudaFree(d_cycles); cudaFree(d_sink); cudaSetDevice(prev); return GIFT_E_INVAL;
     }
     int rc = GIFT_OK;
@@ -166,7 +173,7 @@ extern "C" int gift_probe_pipe(int device, int kind, uint32_t iters, double* lan
         for (int i = 0; i < sms; i++) mean += (double)h[i];
         mean /= sms;
         delete[] h;
-        static const double per_step[18] = {1, 1, 1, 1, 1, 1, 2, 1, 2, 1, 2, 2, 2, 2, 2, 3, 2, 2};
+        static const double per_step[20] = {1, 1, 1, 1, 1, 1, 2, 1, 2, 1, 2, 2, 2, 2, 2, 3, 2, 2, 1, 2};
         const double per_pair = per_step[kind];                       // instructions per step
         const double ops = 1024.0 * CHAINS * UNROLL * (double)iters * per_pair;
         *lane_ops_per_clk_per_sm = ops / mean;
