@@ -346,7 +346,18 @@ def main():
             dec_ms = timed(lambda: ctx.tok_decrypt(c16, own, 2, t_out, stt), n=20)
             tok["%d_tokens" % nt] = {"encrypt_us": enc_ms * 1e3, "decrypt_us": dec_ms * 1e3,
                                      "encrypt_mtok_s": nt / enc_ms / 1e3, "round_trip_ok": bool(torch.equal(t_out, t_in))}
+        # launch-order check (paper sec. 4.4) over a seeded trace of 20 000 launches on 4 streams
+        tr = W.launch_trace(20000, 4096, 4, race_frac=0.05)
+        sp, se, sw = W.trace_by_segment(tr["acc_ptr"], tr["acc_seg"], tr["acc_write"], 4096)
+        dk, ds = torch.from_numpy(tr["kind"]).cuda(), torch.from_numpy(tr["stream"]).cuda()
+        dsp, dse, dsw = torch.from_numpy(sp).cuda(), torch.from_numpy(se).cuda(), torch.from_numpy(sw).cuda()
+        fl = torch.zeros(len(tr["kind"]), dtype=torch.int32, device="cuda")
+        sm = torch.zeros(2, dtype=torch.int32, device="cuda")
+        order_ms = timed(lambda: ctx.check_launch_order(dk, ds, dsp, dse, dsw, 4, fl, sm), n=20)
+        order = {"events": int(len(tr["kind"])), "accesses": int(len(se)), "check_us": order_ms * 1e3,
+                 "flagged": int(sm[0].item())}
         line["extra"] = {"verify_gbs": payload / ver / 1e6, "verify_all_ok": bool(ok_verify), "token_mode": tok,
+                         "launch_order_check": order,
                          "encrypt_plus_decrypt_gbs": 2 * payload / dec / 1e6,
                          "decrypt_restores_ok": bool(not status.any().item()),
                          "identity_rule_us": rule_us}

@@ -254,6 +254,36 @@ typedef struct {
 int gift_propagate_labels(gift_ctx* ctx, const gift_rule* rule, const int32_t* const* in_owner_maps,
                           int32_t* out_owner_map, uint32_t* viol, void* stream);
 
+/* Multi-stream launch-order check (paper sec. 4.4, "Concurrency control"): the ownership
+ * record of a segment is extended with its last writer kernel and last reader kernels, each
+ * a (stream, sequence) pair, and a kernel counts as completed once a synchronisation of its
+ * stream follows its launch.  A reader of M may launch only if M's last writer, when on
+ * another stream, has completed; a writer of M only if M's last readers and last writer on
+ * other streams have completed.  This call checks a whole recorded trace at once.
+ *   kind[e]    0 kernel launch, 1 synchronisation of stream[e]      (device, n_events)
+ *   stream[e]  stream id in [0, n_streams), n_streams <= 32         (device, n_events)
+ *   seg_ptr / seg_event / seg_write: for every memory segment, the launches that access
+ *   it in launch order (the history its record accumulates): event index and 0 read /
+ *   1 write (device; seg_ptr has n_segments + 1 entries).  A launch that reads and writes
+ *   a segment appears twice, adjacent.
+ * flags[e] (device, n_events) receives GIFT_RACE_* bits for every launch that breaks an
+ * invariant (the monitor would have held it back); the records advance as if it had run.
+ * summary[0] = number of flagged launches, summary[1] = first flagged event or 0xFFFFFFFF.
+ * The struct is host memory; the call may grow a scratch array (synchronises then). */
+#define GIFT_RACE_RAW 1u   /* reads a segment whose last writer on another stream is in flight */
+#define GIFT_RACE_WAR 2u   /* writes a segment that a reader on another stream may still read */
+#define GIFT_RACE_WAW 4u   /* writes a segment whose last writer on another stream is in flight */
+typedef struct {
+    uint32_t n_events, n_streams, n_segments;
+    const uint8_t* kind;
+    const int32_t* stream;
+    const int32_t* seg_ptr;
+    const int32_t* seg_event;
+    const uint8_t* seg_write;
+} gift_trace;
+int gift_check_launch_order(gift_ctx* ctx, const gift_trace* trace, uint32_t* flags, uint32_t* summary,
+                            void* stream);
+
 /* Text for a GIFT_E_* code; never NULL. */
 const char* gift_strerror(int code);
 

@@ -24,7 +24,7 @@ STATIC_MAX_SEGS = 65536
 EXPORTS = [
     "gift_ctx_create", "gift_ctx_destroy", "gift_ctx_reserve", "gift_set_keys", "gift_clear_keys",
     "gift_seg_encrypt", "gift_seg_encrypt_static", "gift_seg_decrypt", "gift_verify_tags",
-    "gift_propagate_labels", "gift_tok_encrypt", "gift_tok_decrypt",
+    "gift_propagate_labels", "gift_tok_encrypt", "gift_tok_decrypt", "gift_check_launch_order",
     "gift_strerror", "gift_version", "gift_launch_count", "gift_timing_enable", "gift_timing_read",
     "gift_probe_pipe",
 ]
@@ -50,6 +50,14 @@ class _Rule(C.Structure):
                 ("seg_ptr", C.c_void_p), ("src_ptr", C.c_void_p), ("src_idx", C.c_void_p),
                 ("gather", C.c_void_p), ("param_mask", C.c_uint32)]
 
+
+class _Trace(C.Structure):
+    _fields_ = [("n_events", C.c_uint32), ("n_streams", C.c_uint32), ("n_segments", C.c_uint32),
+                ("kind", C.c_void_p), ("stream", C.c_void_p), ("seg_ptr", C.c_void_p),
+                ("seg_event", C.c_void_p), ("seg_write", C.c_void_p)]
+
+
+RACE_RAW, RACE_WAR, RACE_WAW = 1, 2, 4
 
 _lib = None
 
@@ -79,6 +87,7 @@ def lib():
                                        C.c_void_p, C.c_void_p, C.c_void_p]
         l.gift_tok_decrypt.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_uint32, C.c_uint64, C.c_void_p,
                                        C.c_void_p, C.c_void_p, C.c_void_p]
+        l.gift_check_launch_order.argtypes = [C.c_void_p, C.POINTER(_Trace), C.c_void_p, C.c_void_p, C.c_void_p]
         l.gift_strerror.restype = C.c_char_p
         l.gift_strerror.argtypes = [C.c_int]
         l.gift_version.restype = C.c_uint32
@@ -230,6 +239,17 @@ class Ctx:
         _check(lib().gift_tok_decrypt(self._h, _dev(in16), _dev(owners), owners.numel(), int(eos_token),
                                       _dev(tokens_out), _dev(nonces_out), _dev(status), _stream_ptr(stream)),
                "gift_tok_decrypt")
+
+    def check_launch_order(self, kind, stream_ids, seg_ptr, seg_event, seg_write, n_streams, flags, summary,
+                           stream=None):
+        import torch
+        if seg_event.numel() == 0:       # no accesses at all: the library still wants valid pointers
+            seg_event = torch.zeros(1, dtype=torch.int32, device=seg_ptr.device)
+            seg_write = torch.zeros(1, dtype=torch.uint8, device=seg_ptr.device)
+        t = _Trace(kind.numel(), n_streams, seg_ptr.numel() - 1, kind.data_ptr(), stream_ids.data_ptr(),
+                   seg_ptr.data_ptr(), seg_event.data_ptr(), seg_write.data_ptr())
+        _check(lib().gift_check_launch_order(self._h, C.byref(t), _dev(flags), _dev(summary), _stream_ptr(stream)),
+               "gift_check_launch_order")
 
     def launch_count(self) -> int:
         return int(lib().gift_launch_count(self._h))

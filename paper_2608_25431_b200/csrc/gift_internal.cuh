@@ -40,6 +40,8 @@ struct gift_ctx {
     uint4* d_acc;                      // [seg_cap]
     uint32_t* d_ticket;                // [seg_cap]
     Globals* d_glob;
+    int32_t* d_next_sync;              // launch-order check: completion time per launch
+    uint32_t order_cap;
     int32_t* d_snapshot;               // label snapshot for aliased rules
     uint32_t snapshot_cap;
     uint64_t launches;

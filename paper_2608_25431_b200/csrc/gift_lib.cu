@@ -779,7 +779,7 @@ int gift_ctx_destroy(gift_ctx* c)
         cudaDeviceSynchronize();
         cudaFree(c->d_t0); cudaFree(c->d_isbox); cudaFree(c->d_hot); cudaFree(c->d_pow); cudaFree(c->d_glob);
         cudaFree(c->d_run_prefix); cudaFree(c->d_acc); cudaFree(c->d_ticket);
-        cudaFree(c->d_stage_ids); cudaFree(c->d_stage_keys); cudaFree(c->d_snapshot);
+        cudaFree(c->d_stage_ids); cudaFree(c->d_stage_keys); cudaFree(c->d_snapshot); cudaFree(c->d_next_sync);
         if (c->h_stage) {
             memset(c->h_stage, 0, (size_t)c->stage_cap * 20);
             cudaFreeHost(c->h_stage);

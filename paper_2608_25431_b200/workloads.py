@@ -316,3 +316,76 @@ def bump_epoch(segs: np.ndarray) -> np.ndarray:
     out = segs.copy()
     out["nonce"][:, 7] ^= 0x80
     return out
+
+
+# --------------------------------------------------------------------------
+# Launch traces for the multi-stream launch-order check (paper sec. 4.4)
+# --------------------------------------------------------------------------
+def launch_trace(n_launches: int = 2000, n_segments: int = 512, n_streams: int = 3, race_frac: float = 0.02,
+                 seed_salt: int = 0):
+    """A seeded trace of kernel launches and synchronisations over n_streams streams.
+
+    Stream 0 is the compute stream: each launch reads a handful of KV-block segments and
+    writes one or two.  The other streams swap KV blocks in the background (one write, or
+    one read, per launch).  A well-behaved framework synchronises a background stream before
+    the compute stream touches what it wrote, and the other way round; with probability
+    race_frac that synchronisation is left out, which plants a race.
+    Returns a dict of numpy arrays: kind, stream (per event), acc_ptr, acc_seg, acc_write.
+    """
+    rng = _rng(6, seed_salt)
+    kind, stream, acc_ptr, acc_seg, acc_write = [], [], [0], [], []
+    dirty = {}          # segment -> (stream, event) of an access not yet synchronised
+
+    def emit_sync(s):
+        kind.append(1)
+        stream.append(s)
+        acc_ptr.append(len(acc_seg))
+        for m in [m for m, (st, _) in dirty.items() if st == s]:
+            del dirty[m]
+
+    def emit_launch(s, reads, writes):
+        for m in list(reads) + list(writes):
+            if m in dirty and dirty[m][0] != s and rng.random() >= race_frac:
+                emit_sync(dirty[m][0])
+        kind.append(0)
+        stream.append(s)
+        for m in reads:
+            acc_seg.append(int(m))
+            acc_write.append(0)
+        for m in writes:
+            acc_seg.append(int(m))
+            acc_write.append(1)
+        acc_ptr.append(len(acc_seg))
+        e = len(kind) - 1
+        for m in list(reads) + list(writes):
+            dirty[int(m)] = (s, e)
+
+    for _ in range(n_launches):
+        if n_streams > 1 and rng.random() < 0.25:
+            s = int(rng.integers(1, n_streams))
+            m = int(rng.integers(0, n_segments))
+            if rng.random() < 0.5:
+                emit_launch(s, [], [m])         # swap in: overwrite a block
+            else:
+                emit_launch(s, [m], [])         # swap out: read a block
+        else:
+            reads = rng.choice(n_segments, size=min(n_segments, int(rng.integers(1, 9))), replace=False)
+            writes = rng.choice(n_segments, size=min(n_segments, int(rng.integers(1, 3))), replace=False)
+            emit_launch(0, reads, writes)
+        if rng.random() < 0.02:
+            emit_sync(int(rng.integers(0, n_streams)))
+    return {"kind": np.array(kind, dtype=np.uint8), "stream": np.array(stream, dtype=np.int32),
+            "acc_ptr": np.array(acc_ptr, dtype=np.int32), "acc_seg": np.array(acc_seg, dtype=np.int32),
+            "acc_write": np.array(acc_write, dtype=np.uint8), "n_streams": n_streams, "n_segments": n_segments}
+
+
+def trace_by_segment(acc_ptr, acc_seg, acc_write, n_segments):
+    """The accesses of a launch trace grouped per segment in launch order (the history that
+    the extended ownership records accumulate): (seg_ptr int32[n_segments+1],
+    seg_event int32[A], seg_write uint8[A]).  A stable sort only; no checking logic."""
+    n_events = len(acc_ptr) - 1
+    ev = np.repeat(np.arange(n_events, dtype=np.int32), np.diff(acc_ptr))
+    order = np.argsort(np.asarray(acc_seg), kind="stable")
+    counts = np.bincount(np.asarray(acc_seg, dtype=np.int64), minlength=n_segments)
+    seg_ptr = np.concatenate([[0], np.cumsum(counts)]).astype(np.int32)
+    return seg_ptr, ev[order].astype(np.int32), np.asarray(acc_write, dtype=np.uint8)[order]
