@@ -284,6 +284,57 @@ typedef struct {
 int gift_check_launch_order(gift_ctx* ctx, const gift_trace* trace, uint32_t* flags, uint32_t* summary,
                             void* stream);
 
+/* Two-level ownership index (paper sec. 4.2, "Ownership data structure"): the first level
+ * maps a base address to a tensor record (base address, shape, element size and the
+ * ownership-related dimensions, e.g. (0) for the rows of a matrix or (0,1,3) of a
+ * 5-dimensional KV tensor); the second level maps the subscripts of those dimensions to an
+ * owner.  A record is host memory; `owners` is a device array with one label per
+ * combination of ownership-related subscripts, row-major. */
+#define GIFT_MAX_DIMS 5
+typedef struct {
+    uint64_t base;
+    uint32_t ndim, elem_size;
+    uint64_t shape[GIFT_MAX_DIMS];
+    uint32_t odim_mask;              /* bit d set: dimension d decides ownership */
+    const int32_t* owners;
+} gift_tensor_rec;
+
+/* One tensor argument of a kernel launch as the framework presents it.  Arguments that
+ * carry the same non-zero alias_group are meant to alias (paper Fig. 6, "Alias" nodes). */
+typedef struct {
+    uint64_t base;
+    uint32_t ndim, alias_group;
+    uint64_t shape[GIFT_MAX_DIMS];
+} gift_kernel_arg;
+
+#define GIFT_ARG_OK       0u
+#define GIFT_ARG_UNKNOWN  1u   /* no record at this base address: memory the monitor does not know (sec. 4.2) */
+#define GIFT_ARG_SHAPE    2u   /* argument shape differs from the record */
+#define GIFT_ARG_ALIAS    4u   /* overlaps another argument without being declared an alias */
+
+/* Steps (1)-(3) of a flow rule (paper sec. 4.3): find each argument's record by base
+ * address, compare shapes, detect unintended aliasing.  Pure host call on host arrays;
+ * rec_of_arg[i] is the record index or -1, arg_status[i] a set of GIFT_ARG_* bits. */
+int gift_resolve_args(const gift_tensor_rec* recs, uint32_t n_rec, const gift_kernel_arg* args, uint32_t n_args,
+                      int32_t* rec_of_arg, uint32_t* arg_status);
+
+/* The contiguous runs of the slice [lo[d], hi[d]) of a recorded tensor (an ownership slice
+ * such as C[1,2,:,0:8,:]), expressed as page numbers in units of the run length counted
+ * from the tensor's base: a paged segment with page_bytes = *run_bytes and these table
+ * entries covers exactly the slice, in row-major order.  Pure host call.  table may be NULL
+ * to query *run_bytes and *n_runs.  GIFT_E_ALIGN when the run length is not a multiple of
+ * 16 bytes or a run does not start on a multiple of it. */
+int gift_slice_runs(const gift_tensor_rec* rec, const uint64_t* lo, const uint64_t* hi, uint64_t* run_bytes,
+                    uint32_t* n_runs, int32_t* table, uint32_t table_cap);
+
+/* Expand the level-2 records of a tensor into one label per run of run_bytes bytes
+ * (unit_owner, device, n_units = tensor bytes / run_bytes): the owner map that the paged
+ * segment calls take.  A run that spans several records (eight slots of a block whose
+ * records are per slot) gets the label they agree on, or GIFT_OWNER_CONFLICT; a run that
+ * is neither a part of one record nor a whole number of records gives GIFT_E_ALIGN. */
+int gift_expand_owners(gift_ctx* ctx, const gift_tensor_rec* rec, uint64_t run_bytes, int32_t* unit_owner,
+                       uint32_t n_units, void* stream);
+
 /* Text for a GIFT_E_* code; never NULL. */
 const char* gift_strerror(int code);
 

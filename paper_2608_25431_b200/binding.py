@@ -25,6 +25,7 @@ EXPORTS = [
     "gift_ctx_create", "gift_ctx_destroy", "gift_ctx_reserve", "gift_set_keys", "gift_clear_keys",
     "gift_seg_encrypt", "gift_seg_encrypt_static", "gift_seg_decrypt", "gift_verify_tags",
     "gift_propagate_labels", "gift_tok_encrypt", "gift_tok_decrypt", "gift_check_launch_order",
+    "gift_resolve_args", "gift_slice_runs", "gift_expand_owners",
     "gift_strerror", "gift_version", "gift_launch_count", "gift_timing_enable", "gift_timing_read",
     "gift_probe_pipe",
 ]
@@ -58,6 +59,63 @@ class _Trace(C.Structure):
 
 
 RACE_RAW, RACE_WAR, RACE_WAW = 1, 2, 4
+ARG_OK, ARG_UNKNOWN, ARG_SHAPE, ARG_ALIAS = 0, 1, 2, 4
+MAX_DIMS = 5
+
+
+class TensorRec(C.Structure):
+    """gift_tensor_rec: base address, shape, element size, ownership-related dimensions, level-2 owners."""
+    _fields_ = [("base", C.c_uint64), ("ndim", C.c_uint32), ("elem_size", C.c_uint32),
+                ("shape", C.c_uint64 * MAX_DIMS), ("odim_mask", C.c_uint32), ("owners", C.c_void_p)]
+
+    @classmethod
+    def make(cls, base, shape, elem_size, odims, owners_ptr=None):
+        r = cls()
+        r.base, r.ndim, r.elem_size = int(base), len(shape), int(elem_size)
+        for d, n in enumerate(shape):
+            r.shape[d] = int(n)
+        r.odim_mask = sum(1 << d for d in odims)
+        r.owners = owners_ptr
+        return r
+
+
+class KernelArg(C.Structure):
+    _fields_ = [("base", C.c_uint64), ("ndim", C.c_uint32), ("alias_group", C.c_uint32),
+                ("shape", C.c_uint64 * MAX_DIMS)]
+
+    @classmethod
+    def make(cls, base, shape, alias_group=0):
+        a = cls()
+        a.base, a.ndim, a.alias_group = int(base), len(shape), int(alias_group)
+        for d, n in enumerate(shape):
+            a.shape[d] = int(n)
+        return a
+
+
+def resolve_args(recs, args):
+    """Steps (1)-(3) of a flow rule on host records: (record index per argument, status bits per argument)."""
+    rarr = (TensorRec * max(1, len(recs)))(*recs)
+    aarr = (KernelArg * max(1, len(args)))(*args)
+    idx = (C.c_int32 * max(1, len(args)))()
+    st = (C.c_uint32 * max(1, len(args)))()
+    f = lib().gift_resolve_args
+    f.argtypes = [C.c_void_p, C.c_uint32, C.c_void_p, C.c_uint32, C.c_void_p, C.c_void_p]
+    _check(f(rarr, len(recs), aarr, len(args), idx, st), "gift_resolve_args")
+    return list(idx)[: len(args)], list(st)[: len(args)]
+
+
+def slice_runs(rec, lo, hi):
+    """(run_bytes, page numbers) of the slice [lo, hi) of a recorded tensor."""
+    lo_a = (C.c_uint64 * MAX_DIMS)(*[int(x) for x in lo])
+    hi_a = (C.c_uint64 * MAX_DIMS)(*[int(x) for x in hi])
+    run, n = C.c_uint64(), C.c_uint32()
+    f = lib().gift_slice_runs
+    f.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_uint32]
+    _check(f(C.byref(rec), lo_a, hi_a, C.byref(run), C.byref(n), None, 0), "gift_slice_runs")
+    table = np.zeros(max(1, n.value), dtype=np.int32)
+    _check(f(C.byref(rec), lo_a, hi_a, C.byref(run), C.byref(n), table.ctypes.data_as(C.c_void_p), table.size),
+           "gift_slice_runs")
+    return run.value, table[: n.value]
 
 _lib = None
 
@@ -250,6 +308,12 @@ class Ctx:
                    seg_ptr.data_ptr(), seg_event.data_ptr(), seg_write.data_ptr())
         _check(lib().gift_check_launch_order(self._h, C.byref(t), _dev(flags), _dev(summary), _stream_ptr(stream)),
                "gift_check_launch_order")
+
+    def expand_owners(self, rec, run_bytes, unit_owner, stream=None):
+        f = lib().gift_expand_owners
+        f.argtypes = [C.c_void_p, C.c_void_p, C.c_uint64, C.c_void_p, C.c_uint32, C.c_void_p]
+        _check(f(self._h, C.byref(rec), int(run_bytes), _dev(unit_owner), unit_owner.numel(), _stream_ptr(stream)),
+               "gift_expand_owners")
 
     def launch_count(self) -> int:
         return int(lib().gift_launch_count(self._h))
