@@ -13,7 +13,7 @@ import os
 import numpy as np
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
-LIB_PATH = os.path.join(_HERE, "libgift.so")
+LIB_PATH = os.environ.get("GIFT_LIB", os.path.join(_HERE, "libgift.so"))
 
 OK, E_INVAL, E_NOMEM, E_CUDA, E_RANGE, E_ALIGN = 0, -1, -2, -3, -4, -5
 ST_TAG_MISMATCH, ST_OWNER_MISMATCH, ST_UNOWNED, ST_NO_KEY, ST_BAD_DESC = 1, 2, 4, 8, 16
