@@ -103,6 +103,7 @@ struct CallArgs {
     uint32_t* ticket;
     Globals* glob;
     uint32_t target_runs;          // runs wanted for a balanced call
+    uint32_t resident_warps;       // warps of the cipher kernel on the whole GPU
     uint32_t max_run_blocks;
     uint32_t min_run_blocks;
 };
@@ -214,11 +215,17 @@ __global__ void scan_kernel(CallArgs a)
     __shared__ uint32_t run_blocks_s;
     const int tid = threadIdx.x, lane = tid & 31, wid = tid >> 5;
     if (tid == 0) {
-        // smallest power of two that keeps the run count near the target, within limits
+        // Run length (a multiple of 32 blocks, so that rows stay aligned): large calls get about
+        // eight runs per resident warp, so that the dynamic hand-out evens out skewed segment
+        // lengths; calls too small for that get one run per warp, which avoids a second,
+        // mostly empty wave.
         const unsigned long long total = a.glob->total_blocks;
-        uint32_t rb = a.min_run_blocks;
-        while (rb < a.max_run_blocks && total / rb > a.target_runs) rb <<= 1;
-        run_blocks_s = rb;
+        unsigned long long rb = (total + a.target_runs - 1) / a.target_runs;
+        if (rb < 512) rb = (total + a.resident_warps - 1) / a.resident_warps;
+        rb = (rb + 31) / 32 * 32;
+        if (rb < a.min_run_blocks) rb = a.min_run_blocks;
+        if (rb > a.max_run_blocks) rb = a.max_run_blocks;
+        run_blocks_s = (uint32_t)rb;
         carry = 0u;
     }
     __syncthreads();
@@ -688,9 +695,10 @@ int seg_call(gift_ctx* c, const void* src, void* dst, uint64_t buf_bytes, const 
     a.acc = c->d_acc;
     a.ticket = c->d_ticket;
     a.glob = c->d_glob;
-    a.target_runs = (uint32_t)c->num_sms * (uint32_t)(c->threads / 32) * 8u;   // about eight runs per resident warp
+    a.resident_warps = (uint32_t)c->num_sms * (uint32_t)(c->threads / 32);
+    a.target_runs = a.resident_warps * 8u;                // about eight runs per resident warp
     a.max_run_blocks = 4096u;                             // 64 KiB
-    a.min_run_blocks = 256u;                              // 4 KiB
+    a.min_run_blocks = 64u;                               // 1 KiB
 
     CU_TRY(cudaMemsetAsync(c->d_glob, 0, sizeof(Globals), st));
     const uint32_t plan_blocks = (nseg + 7) / 8;          // 8 warps per block, one warp per segment
@@ -1088,9 +1096,10 @@ extern "C" int gift_seg_encrypt_static(gift_ctx* c, const void* src, void* dst, 
     a.run_prefix = reinterpret_cast<uint32_t*>(scratch + STATIC_OFF_PREFIX);
     a.acc = reinterpret_cast<uint4*>(scratch + STATIC_OFF_ACC);
     a.ticket = reinterpret_cast<uint32_t*>(scratch + STATIC_OFF_TICKET);
-    a.target_runs = (uint32_t)c->num_sms * (uint32_t)(c->threads / 32) * 8u;
+    a.resident_warps = (uint32_t)c->num_sms * (uint32_t)(c->threads / 32);
+    a.target_runs = a.resident_warps * 8u;
     a.max_run_blocks = 4096u;
-    a.min_run_blocks = 256u;
+    a.min_run_blocks = 64u;
 
     // The array still holds the previous call's values: the counters are cleared here, the
     // per-segment accumulators and tickets by the plan kernel, the work list by the scan kernel.
