@@ -244,4 +244,46 @@ GIFT_HD void ctr_keystream(const Tab& tb, const uint32_t* rk, const CtrPrefix& p
     aes_last_round(tb, ks, rk + 40);
 }
 
+// ---- CTR across 256 consecutive counters ----
+//
+// Inside a group of 256 consecutive counter values only the counter's lowest byte changes,
+// which is byte 3 of the varying state word.  After round 1 only column 0 depends on it;
+// in round 2 every output column takes exactly one byte of column 0, so three of its four
+// lookups are the same for the whole group.  `CtrGroup` caches what is constant per group:
+// the round-2 constants.  Per block that leaves 1 lookup in round 1 and 4 in round 2.
+struct CtrGroup {
+    uint32_t grp;      // ctr >> 8 the cache belongs to
+    uint32_t c2[4];    // round-2 output column c without the lookup that depends on column 0
+};
+
+template <class Tab>
+GIFT_HD void ctr_group_setup(const Tab& tb, const uint32_t* rk, const CtrPrefix& p, uint32_t ctr, CtrGroup& g)
+{
+    const uint32_t d = bswap32(ctr) ^ p.k03;                 // bytes 0..2 are what the group shares
+    const uint32_t k1 = p.c1[1] ^ tb.template look<2, 2>(d);  // round-1 columns 1..3
+    const uint32_t k2 = p.c1[2] ^ tb.template look<1, 1>(d);
+    const uint32_t k3 = p.c1[3] ^ tb.template look<0, 0>(d);
+    g.grp = ctr >> 8;
+    g.c2[0] = tb.template look<1, 1>(k1) ^ tb.template look<2, 2>(k2) ^ tb.template look<3, 3>(k3) ^ rk[8];
+    g.c2[1] = tb.template look<0, 0>(k1) ^ tb.template look<1, 1>(k2) ^ tb.template look<2, 2>(k3) ^ rk[9];
+    g.c2[2] = tb.template look<0, 0>(k2) ^ tb.template look<1, 1>(k3) ^ tb.template look<3, 3>(k1) ^ rk[10];
+    g.c2[3] = tb.template look<0, 0>(k3) ^ tb.template look<2, 2>(k1) ^ tb.template look<3, 3>(k2) ^ rk[11];
+}
+
+// Keystream block for counter value ctr, which must lie in the group g was set up for.
+template <class Tab>
+GIFT_HD void ctr_keystream_grouped(const Tab& tb, const uint32_t* rk, const CtrPrefix& p, const CtrGroup& g,
+                                   uint32_t ctr, uint32_t ks[4])
+{
+    const uint32_t d = bswap32(ctr) ^ p.k03;
+    const uint32_t x0 = p.c1[0] ^ tb.template look<3, 3>(d);          // round 1, column 0
+    ks[0] = g.c2[0] ^ tb.template look<0, 0>(x0);                      // round 2
+    ks[1] = g.c2[1] ^ tb.template look<3, 3>(x0);
+    ks[2] = g.c2[2] ^ tb.template look<2, 2>(x0);
+    ks[3] = g.c2[3] ^ tb.template look<1, 1>(x0);
+#pragma unroll
+    for (int r = 3; r < 10; r++) aes_round(tb, ks, rk + 4 * r);
+    aes_last_round(tb, ks, rk + 40);
+}
+
 }  // namespace gift

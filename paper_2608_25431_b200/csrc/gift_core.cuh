@@ -242,13 +242,18 @@ GIFT_HD u128 run_lane_rows(const Tab& tb, const uint32_t* rk, const CtrPrefix& p
     Block c_prev;
     c_prev.d[0] = c_prev.d[1] = c_prev.d[2] = c_prev.d[3] = 0;
     bool pending = false;
+    CtrGroup grp;
+    grp.grp = ~(ctr >> 8);                                  // forces the first set-up
+    grp.c2[0] = grp.c2[1] = grp.c2[2] = grp.c2[3] = 0;
 #pragma unroll 1
     for (uint32_t j = 0; j < rows; j++) {
         const Block d = load_block(src + off);
         Block c = d;
         if (MODE != MODE_VERIFY) {
             uint32_t ks[4];
-            ctr_keystream(tb, rk, pre, ctr, ks);
+            // the counter advances by 32 per row: a lane enters a new group of 256 every 8 rows
+            if ((ctr >> 8) != grp.grp) ctr_group_setup(tb, rk, pre, ctr, grp);
+            ctr_keystream_grouped(tb, rk, pre, grp, ctr, ks);
             Block o;
             o.d[0] = d.d[0] ^ ks[0]; o.d[1] = d.d[1] ^ ks[1];
             o.d[2] = d.d[2] ^ ks[2]; o.d[3] = d.d[3] ^ ks[3];
