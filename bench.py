@@ -36,11 +36,11 @@ UNIT = "GB/s"
 # DRAM bytes per payload byte of the cipher kernel, from the ncu capture summarised in
 # profiles/crypt_kernel_c3_2layers.md (dram__bytes_read.sum + dram__bytes_write.sum over the
 # payload of that launch); traffic grows in proportion to the payload.
-NCU_DRAM_BYTES_PER_PAYLOAD_BYTE = 1.926
+NCU_DRAM_BYTES_PER_PAYLOAD_BYTE = 1.931
 
 # ALU-pipe instructions per block the cipher kernel actually executes (ncu, same capture):
 # the tighter ceiling "if this very instruction stream issued at the pipe's full rate".
-EXECUTED_ALU_OPS_PER_BLOCK = 489
+EXECUTED_ALU_OPS_PER_BLOCK = 483
 
 ALU_OPS_PER_BLOCK = 660          # logic / permute / shift / add lane-operations
 MUL_OPS_PER_BLOCK = 144          # 32x32 -> 64 multiplies
