@@ -30,21 +30,19 @@ if ROOT not in sys.path:
 METRIC = "segment encrypt+tag throughput"
 UNIT = "GB/s"
 
-# Integer work per 16-byte block of the best formulation known to this build (frozen; the
-# kernel's own instruction count is not used): T-table AES-CTR with the first round hoisted
-# and GHASH by masked integer multiplies with two Karatsuba levels.
-# DRAM bytes per payload byte of the cipher kernel, from the ncu capture summarised in
-# profiles/crypt_kernel_c3_2layers.md (dram__bytes_read.sum + dram__bytes_write.sum over the
-# payload of that launch); traffic grows in proportion to the payload.
-NCU_DRAM_BYTES_PER_PAYLOAD_BYTE = 1.931
-
-# ALU-pipe instructions per block the cipher kernel actually executes (ncu, same capture):
-# the tighter ceiling "if this very instruction stream issued at the pipe's full rate".
-EXECUTED_ALU_OPS_PER_BLOCK = 483
-
-ALU_OPS_PER_BLOCK = 660          # logic / permute / shift / add lane-operations
-MUL_OPS_PER_BLOCK = 144          # 32x32 -> 64 multiplies
-LDS_OPS_PER_BLOCK = 150          # 4-byte shared-memory lookups
+# Integer work per 16-byte block.  The operation budget this build started from (T-table
+# AES-CTR with the first round hoisted, GHASH by masked integer multiplies with two Karatsuba
+# levels) was 660 logic-pipe operations, 144 wide multiplies and 150 shared-memory lookups.
+# Cheaper formulations were found since (one-instruction table addressing with four tables,
+# class merges as multiply-adds, round-2 constants cached per 256 counters), so the budget
+# was LOWERED, which raises the ceiling: the figures below are what the best formulation
+# known to this build needs on each pipe (they equal what the kernel executes, by ncu).
+# `roofline.frac` uses the lowered budget; `frac_first_budget` is kept for comparison.
+FIRST_ALU_OPS_PER_BLOCK = 660
+ALU_OPS_PER_BLOCK = 483          # logic / permute / shift lane-operations (the binding pipe)
+MUL_OPS_PER_BLOCK = 230          # multiply-pipe lane-operations: 144 wide multiplies + multiply-adds
+LDS_OPS_PER_BLOCK = 176          # shared-memory lane-loads (table lookups, key material)
+ALL_OPS_PER_BLOCK = 901          # every issued lane-instruction
 
 
 def build_workload(name: str, layers: int):
@@ -285,7 +283,7 @@ def main():
     t_alu = ALU_OPS_PER_BLOCK * nblk / (sms * r_alu * f)
     t_mul = MUL_OPS_PER_BLOCK * nblk / (sms * r_mul * f)
     t_lds = LDS_OPS_PER_BLOCK * nblk / (sms * r_lds * f)
-    t_issue = (ALU_OPS_PER_BLOCK + MUL_OPS_PER_BLOCK + LDS_OPS_PER_BLOCK) * nblk / (sms * r_issue * f)
+    t_issue = ALL_OPS_PER_BLOCK * nblk / (sms * r_issue * f)
     t_hbm = (2.0 * payload + 56.0 * nseg) / (hbm_gbs * 1e9)
     t_roof = max(t_alu, t_mul, t_lds, t_issue, t_hbm)
     achieved_tops = ALU_OPS_PER_BLOCK * nblk / (kern_ms * 1e-3) / 1e12
@@ -300,8 +298,9 @@ def main():
                 "ceilings_gbs": {"alu": payload / t_alu / 1e9, "mul": payload / t_mul / 1e9,
                                  "lds": payload / t_lds / 1e9, "issue": payload / t_issue / 1e9,
                                  "hbm": payload / t_hbm / 1e9},
-                "frac_vs_executed_alu": (EXECUTED_ALU_OPS_PER_BLOCK * nblk / (sms * r_alu * f)) / (kern_ms * 1e-3),
-                "executed_alu_ops_per_block": EXECUTED_ALU_OPS_PER_BLOCK,
+                "frac_first_budget": (FIRST_ALU_OPS_PER_BLOCK * nblk / (sms * r_alu * f)) / (kern_ms * 1e-3),
+                "budget_per_block": {"alu": ALU_OPS_PER_BLOCK, "mul": MUL_OPS_PER_BLOCK, "lds": LDS_OPS_PER_BLOCK,
+                                     "all": ALL_OPS_PER_BLOCK, "first_alu": FIRST_ALU_OPS_PER_BLOCK},
                 "sm_mhz_used": f_mhz,
                 "peak_source": "148 SMs x 64 integer lanes x sampled SM clock; HBM from MEASURED_PEAKS.json (of measured)"
                 if peaks else "fallback HBM 6650 GB/s (of fallback)"}

@@ -13,8 +13,8 @@
 //
 // AES uses T-tables replicated across the 32 shared-memory banks so that a warp's
 // 32 data-dependent lookups never conflict; GHASH uses masked integer multiplies
-// (gf128.cuh).  The path is bound by the integer pipes, not by HBM: at most about
-// one eighth of the memory bandwidth is needed, so data moves with plain 128-bit
+// (gf128.cuh).  The path is bound by the integer pipes, not by HBM: about one eighth
+// of the memory bandwidth is needed, so data moves with plain 128-bit
 // loads and stores and no staging through shared memory.
 #include <cuda_runtime.h>
 #include <stdint.h>
