@@ -357,7 +357,7 @@ int gift_timing_read(gift_ctx* ctx, double* total_ms, uint32_t* launches);
  * the SM clock seen.  kind: 0 three-input logic, 1 32x32+64 wide multiply-add, 2 byte
  * permute, 3 conflict-free shared-memory load, 4 funnel shift, 5 integer add, 6 logic and
  * wide multiply interleaved, 7 32-bit multiply-add, 8 logic and shared loads interleaved,
- * 9-19 further kinds and pairings (wide multiply without accumulate, logic with 32-bit multiply-add,
+ * 9-19 further kinds and pairings, 20-32 instruction mixes like the cipher kernel's (wide multiply without accumulate, logic with 32-bit multiply-add,
  * with add, with permute, permute or shared load with wide multiply, and so on).
  * Host call; allocates a few KB, synchronises. */
 int gift_probe_pipe(int device, int kind, uint32_t iters, double* lane_ops_per_clk_per_sm, double* sm_mhz);

@@ -331,7 +331,12 @@ class Ctx:
 PROBE_KINDS = {0: "lop3", 1: "mad.wide.u32", 2: "prmt", 3: "ld.shared.u32", 4: "shf", 5: "add.u32",
                6: "lop3+mad.wide", 7: "mad.lo.u32", 8: "lop3+ld.shared", 9: "mul.wide.u32",
                10: "lop3+mul.wide", 11: "lop3+mad.lo", 12: "lop3+add", 13: "prmt+mad.wide",
-               14: "lop3(imm)+mad.wide", 15: "2 lop3+mad.wide", 16: "ld.shared+mad.wide", 17: "lop3+prmt", 18: "mul.hi.u32", 19: "lop3+mul.hi"}
+               14: "lop3(imm)+mad.wide", 15: "2 lop3+mad.wide", 16: "ld.shared+mad.wide", 17: "lop3+prmt", 18: "mul.hi.u32", 19: "lop3+mul.hi",
+               20: "cipher mix (15 logic, 5 multiply, 4 lookups per 24)", 21: "2 lop3+mul.wide",
+               22: "lop3+prmt+mul.wide", 23: "3 lop3+ld.shared", 24: "2 lop3+mul.wide+ld.shared+xor",
+               25: "2 lop3 (low half)+mul.wide", 26: "2 lop3 (high half)+mul.wide", 27: "2 lop3+mad.lo",
+               28: "3 lop3+mul.wide", 29: "lop3(low,high)+lop3+mul.wide", 30: "mad.lo(high)+2 lop3+mul.wide",
+               31: "prmt(high)+lop3+mul.wide", 32: "mul.wide, 4 lop3, lop3(high)"}
 
 
 def probe_pipe(kind: int, iters: int = 2000, device: int = 0):

@@ -62,14 +62,14 @@ __global__ void __launch_bounds__(1024, 1) probe_kernel(uint32_t iters, uint32_t
                 } else if (KIND == 9) {   // 32x32 -> 64 multiply without accumulate
                     asm volatile("mul.wide.u32 %0, %1, %2;" : "=l"(w[c]) : "r"(x[c]), "r"(k1));
                 } else if (KIND == 10) {  // logic + wide multiply without accumulate
-                    asm volatile("lop3.b32 %0, %0, %1, %2, 0x96;" : "+r"(x[c]) : "r"(k1), "r"(k2));
-                    asm volatile("mul.wide.u32 %0, %1, %2;" : "=l"(w[c]) : "r"(k2), "r"(k1));
+                    asm volatile("lop3.b32 %0, %0, %1, %2, 0x96;" : "+r"(x[c]) : "r"(k1), "r"((uint32_t)w[c]));
+                    asm volatile("mul.wide.u32 %0, %1, %2;" : "=l"(w[c]) : "r"(x[c]), "r"(k1));
                 } else if (KIND == 11) {  // logic + 32-bit multiply-add
-                    asm volatile("lop3.b32 %0, %0, %1, %2, 0x96;" : "+r"(x[c]) : "r"(k1), "r"(k2));
-                    asm volatile("mad.lo.u32 %0, %1, %2, %3;" : "=r"(*reinterpret_cast<uint32_t*>(&w[c])) : "r"(k2), "r"(k1), "r"(k2));
+                    asm volatile("lop3.b32 %0, %0, %1, %2, 0x96;" : "+r"(x[c]) : "r"(k1), "r"((uint32_t)w[c]));
+                    asm volatile("mad.lo.u32 %0, %1, %2, %3;" : "=r"(*reinterpret_cast<uint32_t*>(&w[c])) : "r"(x[c]), "r"(k1), "r"(k2));
                 } else if (KIND == 12) {  // logic + add
-                    asm volatile("lop3.b32 %0, %0, %1, %2, 0x96;" : "+r"(x[c]) : "r"(k1), "r"(k2));
-                    asm volatile("add.u32 %0, %1, %2;" : "=r"(*reinterpret_cast<uint32_t*>(&w[c])) : "r"(k2), "r"(k1));
+                    asm volatile("lop3.b32 %0, %0, %1, %2, 0x96;" : "+r"(x[c]) : "r"(k1), "r"((uint32_t)w[c]));
+                    asm volatile("add.u32 %0, %1, %2;" : "=r"(*reinterpret_cast<uint32_t*>(&w[c])) : "r"(x[c]), "r"(k1));
                 } else if (KIND == 13) {  // byte permute + wide multiply-add
                     asm volatile("prmt.b32 %0, %0, %1, 0x2103;" : "+r"(x[c]) : "r"(k1));
                     asm volatile("mad.wide.u32 %0, %1, %2, %0;" : "+l"(w[c]) : "r"(k2), "r"(k1));
@@ -89,8 +89,83 @@ __global__ void __launch_bounds__(1024, 1) probe_kernel(uint32_t iters, uint32_t
                 } else if (KIND == 18) {  // high half of a 32x32 multiply
                     asm volatile("mul.hi.u32 %0, %0, %1;" : "+r"(x[c]) : "r"(k1));
                 } else if (KIND == 19) {  // logic + high-half multiply
+                    asm volatile("lop3.b32 %0, %0, %1, %2, 0x96;" : "+r"(x[c]) : "r"(k1), "r"((uint32_t)w[c]));
+                    asm volatile("mul.hi.u32 %0, %1, %2;" : "=r"(*reinterpret_cast<uint32_t*>(&w[c])) : "r"(x[c]), "r"(k1));
+                } else if (KIND == 20) {  // the cipher kernel's mix: 11 logic, 3 wide multiplies, 2 multiply-adds, 4 lookups
                     asm volatile("lop3.b32 %0, %0, %1, %2, 0x96;" : "+r"(x[c]) : "r"(k1), "r"(k2));
-                    asm volatile("mul.hi.u32 %0, %1, %2;" : "=r"(*reinterpret_cast<uint32_t*>(&w[c])) : "r"(k2), "r"(k1));
+                    asm volatile("prmt.b32 %0, %0, %1, 0x2103;" : "+r"(x[c]) : "r"(k1));
+                    asm volatile("mul.wide.u32 %0, %1, %2;" : "=l"(w[c]) : "r"(x[c]), "r"(k1));
+                    asm volatile("lop3.b32 %0, %0, %1, %2, 0x69;" : "+r"(x[c]) : "r"(k2), "r"(k1));
+                    x[c] ^= vtab[(x[c] & 2016u) + lane4];
+                    asm volatile("prmt.b32 %0, %0, %1, 0x1032;" : "+r"(x[c]) : "r"(k2));
+                    asm volatile("lop3.b32 %0, %0, %1, %2, 0x96;" : "+r"(x[c]) : "r"((uint32_t)w[c]), "r"(k2));
+                    asm volatile("mad.lo.u32 %0, %0, %1, %2;" : "+r"(x[c]) : "r"(k1), "r"(k2));
+                    asm volatile("prmt.b32 %0, %0, %1, 0x0321;" : "+r"(x[c]) : "r"(k1));
+                    x[c] ^= vtab[(x[c] & 2016u) + lane4];
+                    asm volatile("mul.wide.u32 %0, %1, %2;" : "=l"(w[c]) : "r"(x[c]), "r"(k2));
+                    asm volatile("lop3.b32 %0, %0, %1, %2, 0x96;" : "+r"(x[c]) : "r"((uint32_t)(w[c] >> 32)), "r"(k1));
+                    asm volatile("prmt.b32 %0, %0, %1, 0x2103;" : "+r"(x[c]) : "r"(k2));
+                    x[c] ^= vtab[(x[c] & 2016u) + lane4];
+                    asm volatile("mul.wide.u32 %0, %1, %2;" : "=l"(w[c]) : "r"(x[c]), "r"(k1));
+                    asm volatile("mad.lo.u32 %0, %0, %1, %2;" : "+r"(x[c]) : "r"(k2), "r"((uint32_t)w[c]));
+                    asm volatile("prmt.b32 %0, %0, %1, 0x1230;" : "+r"(x[c]) : "r"(k1));
+                    x[c] ^= vtab[(x[c] & 2016u) + lane4];
+                } else if (KIND == 21) {  // two logic + one wide multiply (no addend)
+                    asm volatile("lop3.b32 %0, %0, %1, %2, 0x96;" : "+r"(x[c]) : "r"(k1), "r"((uint32_t)w[c]));
+                    asm volatile("lop3.b32 %0, %0, %1, %2, 0x69;" : "+r"(x[c]) : "r"(k2), "r"((uint32_t)(w[c] >> 32)));
+                    asm volatile("mul.wide.u32 %0, %1, %2;" : "=l"(w[c]) : "r"(x[c]), "r"(k1));
+                } else if (KIND == 22) {  // logic + permute + wide multiply
+                    asm volatile("lop3.b32 %0, %0, %1, %2, 0x96;" : "+r"(x[c]) : "r"(k1), "r"((uint32_t)w[c]));
+                    asm volatile("prmt.b32 %0, %0, %1, 0x2103;" : "+r"(x[c]) : "r"((uint32_t)(w[c] >> 32)));
+                    asm volatile("mul.wide.u32 %0, %1, %2;" : "=l"(w[c]) : "r"(x[c]), "r"(k1));
+                } else if (KIND == 23) {  // three logic + one independent shared load
+                    asm volatile("lop3.b32 %0, %0, %1, %2, 0x96;" : "+r"(x[c]) : "r"(k1), "r"(k2));
+                    asm volatile("lop3.b32 %0, %0, %1, %2, 0x69;" : "+r"(x[c]) : "r"(k2), "r"(k1));
+                    asm volatile("lop3.b32 %0, %0, %1, %2, 0x96;" : "+r"(x[c]) : "r"(k1), "r"(k1));
+                    w[c] = vtab[lane4 + (c << 5)];
+                } else if (KIND == 24) {  // two logic + one multiply-add + one independent shared load
+                    asm volatile("lop3.b32 %0, %0, %1, %2, 0x96;" : "+r"(x[c]) : "r"(k1), "r"((uint32_t)w[c]));
+                    asm volatile("mul.wide.u32 %0, %1, %2;" : "=l"(w[c]) : "r"(x[c]), "r"(k1));
+                    asm volatile("lop3.b32 %0, %0, %1, %2, 0x69;" : "+r"(x[c]) : "r"(k2), "r"((uint32_t)(w[c] >> 32)));
+                    x[c] ^= vtab[lane4 + (c << 5)];
+                } else if (KIND == 25) {  // as 21, but both logic operations read the low half of the product
+                    asm volatile("lop3.b32 %0, %0, %1, %2, 0x96;" : "+r"(x[c]) : "r"(k1), "r"((uint32_t)w[c]));
+                    asm volatile("lop3.b32 %0, %0, %1, %2, 0x69;" : "+r"(x[c]) : "r"(k2), "r"((uint32_t)w[c]));
+                    asm volatile("mul.wide.u32 %0, %1, %2;" : "=l"(w[c]) : "r"(x[c]), "r"(k1));
+                } else if (KIND == 26) {  // as 21, but only the high half of the product is read
+                    asm volatile("lop3.b32 %0, %0, %1, %2, 0x96;" : "+r"(x[c]) : "r"(k1), "r"(k2));
+                    asm volatile("lop3.b32 %0, %0, %1, %2, 0x69;" : "+r"(x[c]) : "r"(k2), "r"((uint32_t)(w[c] >> 32)));
+                    asm volatile("mul.wide.u32 %0, %1, %2;" : "=l"(w[c]) : "r"(x[c]), "r"(k1));
+                } else if (KIND == 27) {  // two logic + one 32-bit multiply-add
+                    asm volatile("lop3.b32 %0, %0, %1, %2, 0x96;" : "+r"(x[c]) : "r"(k1), "r"((uint32_t)w[c]));
+                    asm volatile("lop3.b32 %0, %0, %1, %2, 0x69;" : "+r"(x[c]) : "r"(k2), "r"(k1));
+                    asm volatile("mad.lo.u32 %0, %1, %2, %3;" : "=r"(*reinterpret_cast<uint32_t*>(&w[c])) : "r"(x[c]), "r"(k1), "r"(k2));
+                } else if (KIND == 28) {  // three logic + one wide multiply
+                    asm volatile("lop3.b32 %0, %0, %1, %2, 0x96;" : "+r"(x[c]) : "r"(k1), "r"((uint32_t)w[c]));
+                    asm volatile("lop3.b32 %0, %0, %1, %2, 0x69;" : "+r"(x[c]) : "r"(k2), "r"(k1));
+                    asm volatile("lop3.b32 %0, %0, %1, %2, 0x96;" : "+r"(x[c]) : "r"(k1), "r"(k1));
+                    asm volatile("mul.wide.u32 %0, %1, %2;" : "=l"(w[c]) : "r"(x[c]), "r"(k1));
+                } else if (KIND == 29) {  // one logic operation reads both halves of the product
+                    asm volatile("lop3.b32 %0, %0, %1, %2, 0x96;" : "+r"(x[c]) : "r"((uint32_t)w[c]), "r"((uint32_t)(w[c] >> 32)));
+                    asm volatile("lop3.b32 %0, %0, %1, %2, 0x69;" : "+r"(x[c]) : "r"(k2), "r"(k1));
+                    asm volatile("mul.wide.u32 %0, %1, %2;" : "=l"(w[c]) : "r"(x[c]), "r"(k1));
+                } else if (KIND == 30) {  // the high half goes through a multiply-add first, logic reads the copy
+                    uint32_t hi2;
+                    asm volatile("mad.lo.u32 %0, %1, %2, %3;" : "=r"(hi2) : "r"((uint32_t)(w[c] >> 32)), "r"(k1), "r"(k2));
+                    asm volatile("lop3.b32 %0, %0, %1, %2, 0x96;" : "+r"(x[c]) : "r"(k1), "r"(hi2));
+                    asm volatile("lop3.b32 %0, %0, %1, %2, 0x69;" : "+r"(x[c]) : "r"(k2), "r"((uint32_t)w[c]));
+                    asm volatile("mul.wide.u32 %0, %1, %2;" : "=l"(w[c]) : "r"(x[c]), "r"(k1));
+                } else if (KIND == 31) {  // the high half read by a permute instead of a logic operation
+                    asm volatile("prmt.b32 %0, %0, %1, 0x2143;" : "+r"(x[c]) : "r"((uint32_t)(w[c] >> 32)));
+                    asm volatile("lop3.b32 %0, %0, %1, %2, 0x69;" : "+r"(x[c]) : "r"(k2), "r"(k1));
+                    asm volatile("mul.wide.u32 %0, %1, %2;" : "=l"(w[c]) : "r"(x[c]), "r"(k1));
+                } else if (KIND == 32) {  // high half read, but two independent logic operations sit between product and use
+                    asm volatile("lop3.b32 %0, %0, %1, %2, 0x96;" : "+r"(x[c]) : "r"(k1), "r"(k2));
+                    asm volatile("lop3.b32 %0, %0, %1, %2, 0x69;" : "+r"(x[c]) : "r"(k2), "r"(k1));
+                    asm volatile("mul.wide.u32 %0, %1, %2;" : "=l"(w[c]) : "r"(x[c]), "r"(k1));
+                    asm volatile("lop3.b32 %0, %0, %1, %2, 0x96;" : "+r"(x[c]) : "r"(k1), "r"(k1));
+                    asm volatile("lop3.b32 %0, %0, %1, %2, 0x69;" : "+r"(x[c]) : "r"(k2), "r"(k2));
+                    asm volatile("lop3.b32 %0, %0, %1, %2, 0x96;" : "+r"(x[c]) : "r"(k1), "r"((uint32_t)(w[c] >> 32)));
                 } else if (KIND == 8) {   // logic and shared-memory loads interleaved
                     asm volatile("lop3.b32 %0, %0, %1, %2, 0x96;" : "+r"(x[c]) : "r"(k1), "r"(k2));
                     w[c] = vtab[lane4 + (c << 5)];
@@ -161,6 +236,19 @@ extern "C" int gift_probe_pipe(int device, int kind, uint32_t iters, double* lan
     case 17: e = run_probe<17>(sms, iters, d_cycles, d_sink, &ms); break;
     case 18: e = run_probe<18>(sms, iters, d_cycles, d_sink, &ms); break;
     case 19: e = run_probe<19>(sms, iters, d_cycles, d_sink, &ms); break;
+    case 20: e = run_probe<20>(sms, iters, d_cycles, d_sink, &ms); break;
+    case 21: e = run_probe<21>(sms, iters, d_cycles, d_sink, &ms); break;
+    case 22: e = run_probe<22>(sms, iters, d_cycles, d_sink, &ms); break;
+    case 23: e = run_probe<23>(sms, iters, d_cycles, d_sink, &ms); break;
+    case 24: e = run_probe<24>(sms, iters, d_cycles, d_sink, &ms); break;
+    case 25: e = run_probe<25>(sms, iters, d_cycles, d_sink, &ms); break;
+    case 26: e = run_probe<26>(sms, iters, d_cycles, d_sink, &ms); break;
+    case 27: e = run_probe<27>(sms, iters, d_cycles, d_sink, &ms); break;
+    case 28: e = run_probe<28>(sms, iters, d_cycles, d_sink, &ms); break;
+    case 29: e = run_probe<29>(sms, iters, d_cycles, d_sink, &ms); break;
+    case 30: e = run_probe<30>(sms, iters, d_cycles, d_sink, &ms); break;
+    case 31: e = run_probe<31>(sms, iters, d_cycles, d_sink, &ms); break;
+    case 32: e = run_probe<32>(sms, iters, d_cycles, d_sink, &ms); break;
     default: cudaFree(d_cycles); cudaFree(d_sink); cudaSetDevice(prev); return GIFT_E_INVAL;
     }
     int rc = GIFT_OK;
@@ -173,7 +261,7 @@ extern "C" int gift_probe_pipe(int device, int kind, uint32_t iters, double* lan
         for (int i = 0; i < sms; i++) mean += (double)h[i];
         mean /= sms;
         delete[] h;
-        static const double per_step[20] = {1, 1, 1, 1, 1, 1, 2, 1, 2, 1, 2, 2, 2, 2, 2, 3, 2, 2, 1, 2};
+        static const double per_step[33] = {1, 1, 1, 1, 1, 1, 2, 1, 2, 1, 2, 2, 2, 2, 2, 3, 2, 2, 1, 2, 24, 3, 3, 4, 5, 3, 3, 3, 4, 3, 4, 3, 6};
         const double per_pair = per_step[kind];                       // instructions per step
         const double ops = 1024.0 * CHAINS * UNROLL * (double)iters * per_pair;
         *lane_ops_per_clk_per_sm = ops / mean;
