@@ -38,6 +38,11 @@ UNIT = "GB/s"
 # was LOWERED, which raises the ceiling: the figures below are what the best formulation
 # known to this build needs on each pipe (they equal what the kernel executes, by ncu).
 # `roofline.frac` uses the lowered budget; `frac_first_budget` is kept for comparison.
+# DRAM bytes per payload byte of the cipher kernel, from the ncu capture summarised in
+# profiles/crypt_kernel_c3_2layers.md (dram__bytes_read.sum + dram__bytes_write.sum over the
+# payload of that launch); traffic grows in proportion to the payload.
+NCU_DRAM_BYTES_PER_PAYLOAD_BYTE = 1.931
+
 FIRST_ALU_OPS_PER_BLOCK = 660
 ALU_OPS_PER_BLOCK = 483          # logic / permute / shift lane-operations (the binding pipe)
 MUL_OPS_PER_BLOCK = 230          # multiply-pipe lane-operations: 144 wide multiplies + multiply-adds
