@@ -373,7 +373,27 @@ def main():
         order_ms = timed(lambda: ctx.check_launch_order(dk, ds, dsp, dse, dsw, 4, fl, sm), n=20)
         order = {"events": int(len(tr["kind"])), "accesses": int(len(se)), "check_us": order_ms * 1e3,
                  "flagged": int(sm[0].item())}
+        # the four flow rules on token owner maps of the mixed batch (config 5 at full size: 131 328 tokens)
+        w5 = W.config5(layers=1, chunk_tokens=512, fill=False)
+        x5 = w5.extra
+        t_own = torch.from_numpy(x5["token_owner"]).cuda()
+        t_out = torch.empty_like(t_own)
+        par = torch.full((1,), binding.OWNER_PARAM, dtype=torch.int32, device="cuda")
+        kv_own = torch.from_numpy(x5["kv_owner"]).cuda()
+        sp5, srcp5 = torch.from_numpy(x5["seg_ptr"]).cuda(), torch.from_numpy(x5["src_ptr"]).cuda()
+        bt5, ga5 = torch.from_numpy(x5["block_table"]).cuda(), torch.from_numpy(x5["gather"]).cuda()
+        rules = {
+            "identity_us": timed(lambda: ctx.propagate_labels(binding.RULE_IDENTITY, [t_own], t_out, viol), n=50) * 1e3,
+            "rowwise_us": timed(lambda: ctx.propagate_labels(binding.RULE_ROWWISE, [t_own, par], t_out, viol,
+                                                             param_mask=2), n=50) * 1e3,
+            "segreduce_us": timed(lambda: ctx.propagate_labels(binding.RULE_SEGREDUCE, [t_own, kv_own], t_out, viol,
+                                                               seg_ptr=sp5, src_ptr=srcp5, src_idx=bt5), n=50) * 1e3,
+            "broadcast_us": timed(lambda: ctx.propagate_labels(binding.RULE_BROADCAST, [t_own], t_out, viol,
+                                                               gather=ga5), n=50) * 1e3,
+            "tokens": int(t_own.numel()), "violations_last": int(viol[0].item()),
+        }
         line["extra"] = {"verify_gbs": payload / ver / 1e6, "verify_all_ok": bool(ok_verify), "token_mode": tok,
+                         "flow_rules": rules,
                          "launch_order_check": order,
                          "encrypt_plus_decrypt_gbs": 2 * payload / dec / 1e6,
                          "decrypt_restores_ok": bool(not status.any().item()),
