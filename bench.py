@@ -392,8 +392,37 @@ def main():
                                                                gather=ga5), n=50) * 1e3,
             "tokens": int(t_own.numel()), "violations_last": int(viol[0].item()),
         }
+        # a decode step's output rows (config 2: 256 rows of 64 004 B): direct calls and a replayed CUDA graph
+        w2 = W.config2()
+        c2 = binding.Ctx(w2.max_users, local, args.flags)
+        c2.set_keys(w2.user_ids, w2.keys)
+        c2.reserve(len(w2.segs))
+        b2 = torch.from_numpy(w2.buf).cuda()
+        s2 = torch.from_numpy(w2.segs.view(np.uint8).copy()).cuda()
+        o2 = torch.from_numpy(w2.owner_map).cuda()
+        tg2 = torch.zeros((len(w2.segs), 16), dtype=torch.uint8, device="cuda")
+        st2 = torch.zeros(len(w2.segs), dtype=torch.int32, device="cuda")
+
+        def rows_call():
+            c2.seg_encrypt(b2, b2, s2, len(w2.segs), tg2, st2, owner_map=o2, unit_bytes=w2.unit_bytes)
+
+        direct_ms = timed(rows_call, n=50)
+        side = torch.cuda.Stream()
+        side.wait_stream(torch.cuda.current_stream())
+        with torch.cuda.stream(side):
+            rows_call()
+        torch.cuda.current_stream().wait_stream(side)
+        torch.cuda.synchronize()
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(graph):
+            rows_call()
+        graph_ms = timed(graph.replay, n=50)
+        decode_rows = {"payload_mb": w2.payload_bytes / 1e6, "direct_us": direct_ms * 1e3, "graph_us": graph_ms * 1e3,
+                       "graph_gbs": w2.payload_bytes / graph_ms / 1e6}
+        del graph
+        c2.close()
         line["extra"] = {"verify_gbs": payload / ver / 1e6, "verify_all_ok": bool(ok_verify), "token_mode": tok,
-                         "flow_rules": rules,
+                         "flow_rules": rules, "decode_rows": decode_rows,
                          "launch_order_check": order,
                          "encrypt_plus_decrypt_gbs": 2 * payload / dec / 1e6,
                          "decrypt_restores_ok": bool(not status.any().item()),
