@@ -344,3 +344,81 @@ def probe_pipe(kind: int, iters: int = 2000, device: int = 0):
     ops, mhz = C.c_double(), C.c_double()
     _check(lib().gift_probe_pipe(device, kind, iters, C.byref(ops), C.byref(mhz)), "gift_probe_pipe")
     return ops.value, mhz.value
+
+
+# ---------------------------------------------------------------------------------------
+# The same calls under the names of include/gift.h, for callers that prefer the C spelling.
+# ---------------------------------------------------------------------------------------
+def gift_ctx_create(max_users: int, device: int = 0, flags: int = 0) -> Ctx:
+    return Ctx(max_users, device, flags)
+
+
+def gift_ctx_destroy(ctx: Ctx):
+    ctx.close()
+
+
+def gift_ctx_reserve(ctx: Ctx, max_segs: int):
+    ctx.reserve(max_segs)
+
+
+def gift_set_keys(ctx: Ctx, user_ids, keys16, stream=None):
+    ctx.set_keys(user_ids, keys16, stream)
+
+
+def gift_clear_keys(ctx: Ctx, user_ids, stream=None):
+    ctx.clear_keys(user_ids, stream)
+
+
+def gift_seg_encrypt(ctx: Ctx, *args, **kw):
+    ctx.seg_encrypt(*args, **kw)
+
+
+def gift_seg_encrypt_static(ctx: Ctx, *args, **kw):
+    ctx.seg_encrypt_static(*args, **kw)
+
+
+def gift_seg_decrypt(ctx: Ctx, *args, **kw):
+    ctx.seg_decrypt(*args, **kw)
+
+
+def gift_verify_tags(ctx: Ctx, *args, **kw):
+    ctx.verify_tags(*args, **kw)
+
+
+def gift_propagate_labels(ctx: Ctx, *args, **kw):
+    ctx.propagate_labels(*args, **kw)
+
+
+def gift_tok_encrypt(ctx: Ctx, *args, **kw):
+    ctx.tok_encrypt(*args, **kw)
+
+
+def gift_tok_decrypt(ctx: Ctx, *args, **kw):
+    ctx.tok_decrypt(*args, **kw)
+
+
+def gift_check_launch_order(ctx: Ctx, *args, **kw):
+    ctx.check_launch_order(*args, **kw)
+
+
+def gift_expand_owners(ctx: Ctx, *args, **kw):
+    ctx.expand_owners(*args, **kw)
+
+
+def gift_timing_enable(ctx: Ctx, on: bool = True):
+    ctx.timing_enable(on)
+
+
+def gift_timing_read(ctx: Ctx):
+    return ctx.timing_read()
+
+
+def gift_launch_count(ctx: Ctx) -> int:
+    return ctx.launch_count()
+
+
+gift_resolve_args = resolve_args
+gift_slice_runs = slice_runs
+gift_probe_pipe = probe_pipe
+gift_strerror = strerror
+gift_version = version

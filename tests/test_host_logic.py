@@ -37,6 +37,8 @@ def test_library_exports_every_declared_symbol():
         assert hasattr(lib, name), name
     from paper_2608_25431_b200 import binding
     assert sorted(binding.EXPORTS) == declared
+    for name in declared:                          # the binding offers every call under its C name
+        assert callable(getattr(binding, name)), name
 
 
 def test_binding_fails_loudly_without_gpu():
