@@ -478,6 +478,23 @@ def main():
                            "mode": "one chunk per layer on 3 streams" if exporter is not None else "one piece",
                            "all_status_clear": ok_e2e}
             if exporter is not None:
+                # the opposite direction: upload ciphertext + tags, decrypt on the device, status words back
+                om_imp = torch.empty_like(om)
+                exporter.import_(h_out, h_tags, buf, chunks, segs, tags, status, h_status, page_table=table,
+                                 page_bytes=w.page_bytes, owner_map=om_imp, unit_bytes=w.unit_bytes)
+                barrier()
+                a.record()
+                for _ in range(k):
+                    exporter.import_(h_out, h_tags, buf, chunks, segs, tags, status, h_status, page_table=table,
+                                     page_bytes=w.page_bytes, owner_map=om_imp, unit_bytes=w.unit_bytes)
+                b.record()
+                barrier()
+                imp_value, imp_ms = replicas.job_throughput(payload, a.elapsed_time(b) / k, "cuda")
+                line["e2e"]["import"] = {"value": imp_value, "unit": UNIT, "ms_per_step": imp_ms,
+                                         "h2d_bytes_per_step": int(w.buf_bytes + nseg * 16),
+                                         "d2h_bytes_per_step": int(nseg * 4),
+                                         "all_status_clear": not bool(h_status.any().item()),
+                                         "plaintext_restored": bool(torch.equal(buf[:1 << 20], h_in[:1 << 20].cuda()))}
                 exporter.close()
             del h_in, h_out
         except RuntimeError as e:

@@ -35,7 +35,12 @@ def layer_chunks(n_layers: int, segs_per_layer: int, bytes_per_layer: int) -> Li
 
 
 class HostExporter:
-    """k contexts and streams that export chunks of a host buffer through one device buffer."""
+    """k contexts and streams that export chunks of a host buffer through one device buffer.
+
+    `import_` is the opposite direction (paper sec. 3, steps 3-4): ciphertext and tags arrive
+    from pinned host memory, every chunk is uploaded and decrypted with the claimed owners'
+    keys on its stream, the plaintext stays on the device and only the status words go back.
+    """
 
     def __init__(self, max_users: int, user_ids, keys, device: int = 0, n_streams: int = 3, flags: int = 0,
                  max_segs_per_chunk: int = 1024):
@@ -80,3 +85,28 @@ class HostExporter:
                 h_status[ch.seg_lo:ch.seg_hi].copy_(d_status[ch.seg_lo:ch.seg_hi], non_blocking=True)
         for st in self.streams:
             cur.wait_stream(st)
+
+    def import_(self, h_src: torch.Tensor, h_tags: torch.Tensor, d_buf: torch.Tensor, chunks: List[Chunk],
+                d_segs: torch.Tensor, d_tags: torch.Tensor, d_status: torch.Tensor, h_status: torch.Tensor,
+                page_table: Optional[torch.Tensor] = None, page_bytes: int = 0,
+                owner_map: Optional[torch.Tensor] = None, unit_bytes: int = 0):
+        """Enqueue upload and in-place decryption of every chunk; returns without waiting."""
+        cur = torch.cuda.current_stream()
+        start = torch.cuda.Event()
+        start.record(cur)
+        for i, ch in enumerate(chunks):
+            st = self.streams[i % len(self.streams)]
+            ctx = self.ctxs[i % len(self.ctxs)]
+            st.wait_event(start)
+            with torch.cuda.stream(st):
+                d_buf[ch.byte_lo:ch.byte_hi].copy_(h_src[ch.byte_lo:ch.byte_hi], non_blocking=True)
+                d_tags[ch.seg_lo:ch.seg_hi].copy_(h_tags[ch.seg_lo:ch.seg_hi], non_blocking=True)
+                n = ch.seg_hi - ch.seg_lo
+                ctx.seg_decrypt(d_buf, d_buf, d_segs[ch.seg_lo * 40: ch.seg_hi * 40], n,
+                                d_tags[ch.seg_lo:ch.seg_hi], d_status[ch.seg_lo:ch.seg_hi],
+                                page_table=page_table, page_bytes=page_bytes, owner_map=owner_map,
+                                unit_bytes=unit_bytes, stream=st.cuda_stream)
+                h_status[ch.seg_lo:ch.seg_hi].copy_(d_status[ch.seg_lo:ch.seg_hi], non_blocking=True)
+        for st in self.streams:
+            cur.wait_stream(st)
+

@@ -40,4 +40,24 @@ def test_layer_chunked_export_matches_oracle():
         assert np.array_equal(h_tags.numpy(), ref_tags)
         assert np.array_equal(h_dst.numpy(), ref)
     assert exp.launch_count() > 0
+    # the way back: upload ciphertext and tags, decrypt on the device, only status words return;
+    # one tampered block must come back as zeros and unowned
+    bad = ref.copy()
+    bad[3 * w.page_bytes + 5] ^= 1
+    victim = int(np.nonzero(w.page_table == 3)[0][0])
+    h_ct = torch.from_numpy(bad).pin_memory()
+    h_tg = torch.from_numpy(ref_tags).pin_memory()
+    om_dev = torch.full((om.size,), -2, dtype=torch.int32, device="cuda")
+    h_status.fill_(9)
+    exp.import_(h_ct, h_tg, d_buf, chunks, d_segs, d_tags, d_status, h_status,
+                page_table=torch.from_numpy(w.page_table).cuda(), page_bytes=w.page_bytes,
+                owner_map=om_dev, unit_bytes=w.unit_bytes)
+    torch.cuda.synchronize()
+    from gpu_harness import oracle_decrypt
+    om_ref = np.full(om.size, -2, dtype=np.int32)
+    pt_ref = bad.copy()
+    st_ref = oracle_decrypt(w, pt_ref, pt_ref, ref_tags, owner_map=om_ref)
+    assert st_ref[victim] == 1 and st_ref[refused] == 1          # the tampered block, and the one never exported
+    assert np.array_equal(h_status.numpy().astype(np.uint32), st_ref)
+    assert np.array_equal(d_buf.cpu().numpy(), pt_ref) and np.array_equal(om_dev.cpu().numpy(), om_ref)
     exp.close()
