@@ -335,6 +335,20 @@ int gift_slice_runs(const gift_tensor_rec* rec, const uint64_t* lo, const uint64
 int gift_expand_owners(gift_ctx* ctx, const gift_tensor_rec* rec, uint64_t run_bytes, int32_t* unit_owner,
                        uint32_t n_units, void* stream);
 
+/* Secure swap space (paper sec. 4.5): KV blocks swapped into the monitor's own memory need
+ * no encryption, but the monitor "tracks ownership of swapped KV blocks" and restores the
+ * records when the blocks come back.  swap_out saves the labels of the listed units
+ * (saved[i] = owner_map[units[i]]) and marks the units GIFT_OWNER_NONE, so that the freed
+ * slots cannot be read; swap_in writes the saved labels to the units the blocks return to,
+ * which need not be the ones they left.  A unit index out of range, or a swap-in onto a
+ * unit that is still owned (it becomes GIFT_OWNER_CONFLICT), is counted in viol[0] with the
+ * smallest offending list position in viol[1] (0xFFFFFFFF if none).  The listed units of
+ * one call must be distinct.  All arrays are device arrays. */
+int gift_labels_swap_out(gift_ctx* ctx, int32_t* owner_map, uint32_t n_units, const int32_t* units, uint32_t n,
+                         int32_t* saved, uint32_t* viol, void* stream);
+int gift_labels_swap_in(gift_ctx* ctx, int32_t* owner_map, uint32_t n_units, const int32_t* units, uint32_t n,
+                        const int32_t* saved, uint32_t* viol, void* stream);
+
 /* Text for a GIFT_E_* code; never NULL. */
 const char* gift_strerror(int code);
 

@@ -81,3 +81,36 @@ def propagate(kind: int, inputs, n_out: int, *, param_mask: int = 0, seg_ptr=Non
     else:
         raise ValueError("unknown rule kind")
     return out, _viol(out)
+
+
+def swap_out(owner_map, units):
+    """Secure swap space (paper sec. 4.5): save the labels of the listed units and unown them.
+
+    Returns (saved int32[n], viol uint32[2]); owner_map is updated in place."""
+    saved = np.empty(len(units), dtype=np.int32)
+    bad = []
+    for i, u in enumerate(units):
+        u = int(u)
+        if u < 0 or u >= len(owner_map):
+            saved[i] = CONFLICT
+            bad.append(i)
+            continue
+        saved[i] = owner_map[u]
+        owner_map[u] = NONE
+    return saved, np.array([len(bad), bad[0] if bad else 0xFFFFFFFF], dtype=np.uint32)
+
+
+def swap_in(owner_map, units, saved):
+    """Put saved labels back at the units the blocks return to; an occupied unit is a violation."""
+    bad = []
+    for i, u in enumerate(units):
+        u = int(u)
+        if u < 0 or u >= len(owner_map):
+            bad.append(i)
+            continue
+        if owner_map[u] != NONE:
+            owner_map[u] = CONFLICT
+            bad.append(i)
+        else:
+            owner_map[u] = saved[i]
+    return np.array([len(bad), bad[0] if bad else 0xFFFFFFFF], dtype=np.uint32)

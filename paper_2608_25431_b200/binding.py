@@ -25,7 +25,7 @@ EXPORTS = [
     "gift_ctx_create", "gift_ctx_destroy", "gift_ctx_reserve", "gift_set_keys", "gift_clear_keys",
     "gift_seg_encrypt", "gift_seg_encrypt_static", "gift_seg_decrypt", "gift_verify_tags",
     "gift_propagate_labels", "gift_tok_encrypt", "gift_tok_decrypt", "gift_check_launch_order",
-    "gift_resolve_args", "gift_slice_runs", "gift_expand_owners",
+    "gift_resolve_args", "gift_slice_runs", "gift_expand_owners", "gift_labels_swap_out", "gift_labels_swap_in",
     "gift_strerror", "gift_version", "gift_launch_count", "gift_timing_enable", "gift_timing_read",
     "gift_probe_pipe",
 ]
@@ -315,6 +315,18 @@ class Ctx:
         _check(f(self._h, C.byref(rec), int(run_bytes), _dev(unit_owner), unit_owner.numel(), _stream_ptr(stream)),
                "gift_expand_owners")
 
+    def labels_swap_out(self, owner_map, units, saved, viol, stream=None):
+        f = lib().gift_labels_swap_out
+        f.argtypes = [C.c_void_p, C.c_void_p, C.c_uint32, C.c_void_p, C.c_uint32, C.c_void_p, C.c_void_p, C.c_void_p]
+        _check(f(self._h, _dev(owner_map), owner_map.numel(), _dev(units), units.numel(), _dev(saved), _dev(viol),
+                 _stream_ptr(stream)), "gift_labels_swap_out")
+
+    def labels_swap_in(self, owner_map, units, saved, viol, stream=None):
+        f = lib().gift_labels_swap_in
+        f.argtypes = [C.c_void_p, C.c_void_p, C.c_uint32, C.c_void_p, C.c_uint32, C.c_void_p, C.c_void_p, C.c_void_p]
+        _check(f(self._h, _dev(owner_map), owner_map.numel(), _dev(units), units.numel(), _dev(saved), _dev(viol),
+                 _stream_ptr(stream)), "gift_labels_swap_in")
+
     def launch_count(self) -> int:
         return int(lib().gift_launch_count(self._h))
 
@@ -403,6 +415,14 @@ def gift_check_launch_order(ctx: Ctx, *args, **kw):
 
 def gift_expand_owners(ctx: Ctx, *args, **kw):
     ctx.expand_owners(*args, **kw)
+
+
+def gift_labels_swap_out(ctx: Ctx, *args, **kw):
+    ctx.labels_swap_out(*args, **kw)
+
+
+def gift_labels_swap_in(ctx: Ctx, *args, **kw):
+    ctx.labels_swap_in(*args, **kw)
 
 
 def gift_timing_enable(ctx: Ctx, on: bool = True):

@@ -70,9 +70,86 @@ __global__ void expand_owners_kernel(ExpandArgs a)
     a.out[u] = label;
 }
 
+// Secure swap space (paper sec. 4.5): blocks swapped to the monitor's own memory are not
+// encrypted, but their ownership travels with them.
+__global__ void swap_out_kernel(int32_t* owner_map, uint32_t n_units, const int32_t* __restrict__ units, uint32_t n,
+                                int32_t* __restrict__ saved, uint32_t* viol)
+{
+    const uint32_t i = blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= n) return;
+    const int32_t u = units[i];
+    if (u < 0 || (uint32_t)u >= n_units) {
+        saved[i] = GIFT_OWNER_CONFLICT;
+        atomicAdd(viol, 1u);
+        atomicMin(viol + 1, i);
+        return;
+    }
+    saved[i] = owner_map[u];
+    owner_map[u] = GIFT_OWNER_NONE;          // the freed slot may not be read (sec. 4.2)
+}
+
+__global__ void swap_in_kernel(int32_t* owner_map, uint32_t n_units, const int32_t* __restrict__ units, uint32_t n,
+                               const int32_t* __restrict__ saved, uint32_t* viol)
+{
+    const uint32_t i = blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= n) return;
+    const int32_t u = units[i];
+    bool bad = u < 0 || (uint32_t)u >= n_units;
+    if (!bad) {
+        // a slot that still holds someone's data must not be overwritten by a swap-in
+        const bool occupied = owner_map[u] != GIFT_OWNER_NONE;
+        owner_map[u] = occupied ? GIFT_OWNER_CONFLICT : saved[i];
+        bad = occupied;
+    }
+    if (bad) {
+        atomicAdd(viol, 1u);
+        atomicMin(viol + 1, i);
+    }
+}
+
+__global__ void swap_viol_init_kernel(uint32_t* viol)
+{
+    viol[0] = 0u;
+    viol[1] = 0xFFFFFFFFu;
+}
+
 }  // namespace
 
 extern "C" {
+
+int gift_labels_swap_out(gift_ctx* c, int32_t* owner_map, uint32_t n_units, const int32_t* units, uint32_t n,
+                         int32_t* saved, uint32_t* viol, void* stream)
+{
+    if (!c || !viol || (n && (!owner_map || !units || !saved))) return GIFT_E_INVAL;
+    DeviceGuard g(c->device);
+    if (!g.ok) return GIFT_E_CUDA;
+    cudaStream_t st = (cudaStream_t)stream;
+    swap_viol_init_kernel<<<1, 1, 0, st>>>(viol);
+    c->launches++;
+    if (n) {
+        swap_out_kernel<<<(n + 255) / 256, 256, 0, st>>>(owner_map, n_units, units, n, saved, viol);
+        c->launches++;
+    }
+    CU_TRY(cudaGetLastError());
+    return GIFT_OK;
+}
+
+int gift_labels_swap_in(gift_ctx* c, int32_t* owner_map, uint32_t n_units, const int32_t* units, uint32_t n,
+                        const int32_t* saved, uint32_t* viol, void* stream)
+{
+    if (!c || !viol || (n && (!owner_map || !units || !saved))) return GIFT_E_INVAL;
+    DeviceGuard g(c->device);
+    if (!g.ok) return GIFT_E_CUDA;
+    cudaStream_t st = (cudaStream_t)stream;
+    swap_viol_init_kernel<<<1, 1, 0, st>>>(viol);
+    c->launches++;
+    if (n) {
+        swap_in_kernel<<<(n + 255) / 256, 256, 0, st>>>(owner_map, n_units, units, n, saved, viol);
+        c->launches++;
+    }
+    CU_TRY(cudaGetLastError());
+    return GIFT_OK;
+}
 
 int gift_resolve_args(const gift_tensor_rec* recs, uint32_t n_rec, const gift_kernel_arg* args, uint32_t n_args,
                       int32_t* rec_of_arg, uint32_t* arg_status)

@@ -147,3 +147,26 @@ def test_config5_rules_tamper_detection_and_reencrypt():
     assert np.array_equal(np.nonzero(ref_st2)[0], x["poisoned"]) and (ref_st2[x["poisoned"]] == 4).all()
     assert not np.array_equal(ref_tags2[good], ref_tags[good])
     ctx.close()
+
+
+def test_swap_space_labels_match_oracle(ctx):
+    rng = np.random.default_rng(23)
+    n_units = 5000
+    om = rng.choice([0, 1, 2, 3, L.NONE, L.PARAM], size=n_units, p=[.2, .2, .2, .2, .15, .05]).astype(np.int32)
+    units = rng.permutation(n_units)[:1200].astype(np.int32)
+    units[7], units[900] = -3, n_units + 4                        # bad list entries
+    d_om, d_units = dev(om), dev(units)
+    saved = torch.full((1200,), 77, dtype=torch.int32, device="cuda")
+    viol = torch.full((2,), 5, dtype=torch.int32, device="cuda")
+    ctx.labels_swap_out(d_om, d_units, saved, viol)
+    torch.cuda.synchronize()
+    ref_om = om.copy()
+    ref_saved, ref_viol = L.swap_out(ref_om, units)
+    assert np.array_equal(np_(saved), ref_saved) and np.array_equal(np_(viol).astype(np.uint32), ref_viol)
+    assert np.array_equal(np_(d_om), ref_om)
+    back = rng.permutation(n_units)[:1200].astype(np.int32)       # they return to other slots, some still occupied
+    ctx.labels_swap_in(d_om, dev(back), saved, viol)
+    torch.cuda.synchronize()
+    ref_viol = L.swap_in(ref_om, back, ref_saved)
+    assert np.array_equal(np_(d_om), ref_om) and np.array_equal(np_(viol).astype(np.uint32), ref_viol)
+    assert ref_viol[0] > 0

@@ -161,3 +161,14 @@ def test_rules_read_a_snapshot_when_aliased():
     m = np.array([0, 1, 2, 3], np.int32)
     out, _ = L.propagate(L.BROADCAST, [m], 4, gather=np.array([3, 2, 1, 0], np.int32))
     assert out.tolist() == [3, 2, 1, 0]
+
+
+def test_swap_space_keeps_ownership_with_the_blocks():
+    om = np.array([0, 0, 1, 1, 2, N, N, N], np.int32)
+    saved, viol = L.swap_out(om, [2, 3, 0])                       # Bob's two blocks and one of Alice's leave
+    assert saved.tolist() == [1, 1, 0] and viol.tolist() == [0, 0xFFFFFFFF]
+    assert om.tolist() == [N, 0, N, N, 2, N, N, N]                # freed slots are unreadable
+    viol = L.swap_in(om, [6, 7, 5], saved)                        # they come back to other slots
+    assert viol.tolist() == [0, 0xFFFFFFFF] and om.tolist() == [N, 0, N, N, 2, 0, 1, 1]
+    viol = L.swap_in(om, [4, 9], np.array([1, 1], np.int32))      # onto a live block, and out of range
+    assert viol.tolist() == [2, 0] and om[4] == C
