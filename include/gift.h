@@ -169,6 +169,16 @@ int gift_seg_encrypt_static(gift_ctx* ctx, const void* src, void* dst, uint64_t 
                             const gift_seg* segs, uint32_t nseg, const gift_pages* pages,
                             const gift_labels* labels, uint8_t* tags_out, uint32_t* status, void* stream);
 
+/* Bind additional authenticated data to the tags (no counterpart in the paper; the AAD of
+ * SP 800-38D).  After this call gift_seg_encrypt, gift_seg_decrypt and gift_verify_tags
+ * authenticate the 16 bytes aad16[16*i .. 16*i+15] (device array, 16-byte aligned, one
+ * entry per segment of the call) together with segment i: a tag then also vouches for,
+ * say, (owner, logical position, epoch), so that a ciphertext block presented under the
+ * right key and nonce but in the wrong role fails verification.  NULL (the initial state)
+ * turns binding off.  The pointer is used by the calls that follow, not copied.
+ * gift_seg_encrypt_static ignores it. */
+int gift_ctx_bind_aad(gift_ctx* ctx, const uint8_t* aad16);
+
 /* Import (paper sec. 3 steps 3-4): decrypt each segment with the CLAIMED
  * owner's key after checking tags_in[i] over the received ciphertext.  On a
  * match dst receives the plaintext and, if labels are given, the covered units

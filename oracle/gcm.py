@@ -134,8 +134,16 @@ def _tables(page_table, page_bytes, owner_map, unit_bytes):
     return pt, npg, om, nu
 
 
+def _aad(aad, n):
+    if aad is None:
+        return None
+    a = np.ascontiguousarray(aad, dtype=np.uint8).reshape(-1)
+    assert a.size == 16 * n
+    return a
+
+
 def seg_encrypt(src, dst, segs, user_ids, keys, max_users, page_table=None, page_bytes=0,
-                owner_map=None, unit_bytes=0):
+                owner_map=None, unit_bytes=0, aad=None):
     """Encrypt every segment of `segs` from src into dst (may be the same array).
 
     Returns (tags uint8[nseg,16], status uint32[nseg]).
@@ -153,14 +161,15 @@ def seg_encrypt(src, dst, segs, user_ids, keys, max_users, page_table=None, page
     rc = f(_p(src), _p(dst), C.c_uint64(src.size), _p(segs), C.c_uint32(n),
            _p(pt) if pt is not None else None, C.c_uint32(npg), C.c_uint64(page_bytes),
            _p(om) if om is not None else None, C.c_uint32(nu), C.c_uint64(unit_bytes),
-           _p(tab), _p(has), C.c_uint32(max_users), _p(tags), _p(status))
+           _p(tab), _p(has), C.c_uint32(max_users), _p(tags), _p(status),
+           _p(_aad(aad, n)) if aad is not None else None)
     if rc != 0:
         raise ValueError("oracle seg_encrypt: bad call (%d)" % rc)
     return tags[:n], status[:n]
 
 
 def seg_decrypt(src, dst, segs, tags, user_ids, keys, max_users, page_table=None, page_bytes=0,
-                owner_map=None, unit_bytes=0, verify_only=False):
+                owner_map=None, unit_bytes=0, verify_only=False, aad=None):
     """Decrypt (or only verify) every segment; owner_map, when given, is updated in place.
 
     Returns status uint32[nseg].
@@ -181,7 +190,8 @@ def seg_decrypt(src, dst, segs, tags, user_ids, keys, max_users, page_table=None
     rc = f(_p(src), _p(dst), C.c_uint64(src.size), _p(segs), C.c_uint32(n),
            _p(pt) if pt is not None else None, C.c_uint32(npg), C.c_uint64(page_bytes),
            _p(om) if om is not None else None, C.c_uint32(nu), C.c_uint64(unit_bytes),
-           _p(tab), _p(has), C.c_uint32(max_users), _p(tg), _p(status), C.c_int(1 if verify_only else 0))
+           _p(tab), _p(has), C.c_uint32(max_users), _p(tg), _p(status), C.c_int(1 if verify_only else 0),
+           _p(_aad(aad, n)) if aad is not None else None)
     if rc != 0:
         raise ValueError("oracle seg_decrypt: bad call (%d)" % rc)
     return status[:n]

@@ -466,13 +466,15 @@ static int env_bad(const seg_env* e)
 /* Export (paper sec. 3 steps 5-6, sec. 4.1 on key selection from the
  * ownership state): a segment is encrypted only if every unit it covers is
  * owned by the claimed owner, who must have a key.  Otherwise its destination
- * bytes are left as they were, its tag is zero and the status says why. */
+ * bytes are left as they were, its tag is zero and the status says why.
+ * aad16, when not NULL, holds 16 bytes of additional authenticated data per
+ * segment (SP 800-38D sec. 7.1). */
 int gift_oracle_seg_encrypt(const uint8_t* src, uint8_t* dst, uint64_t buf_bytes,
                             const oracle_seg* segs, uint32_t nseg,
                             const int32_t* page_table, uint32_t n_pages, uint64_t page_bytes,
                             const int32_t* owner_map, uint32_t n_units, uint64_t unit_bytes,
                             const uint8_t* keys, const uint8_t* has_key, uint32_t max_users,
-                            uint8_t* tags_out, uint32_t* status)
+                            uint8_t* tags_out, uint32_t* status, const uint8_t* aad16)
 {
     seg_env e = { src, dst, buf_bytes, page_table, n_pages, page_bytes,
                   (int32_t*)owner_map, n_units, unit_bytes, keys, has_key, max_users };
@@ -499,8 +501,8 @@ int gift_oracle_seg_encrypt(const uint8_t* src, uint8_t* dst, uint64_t buf_bytes
         uint8_t* tmp = (uint8_t*)malloc(s->len ? s->len : 1);
         if (!tmp) { failed = 1; continue; }
         seg_gather(&e, s, src, tmp);
-        gift_oracle_gcm_encrypt(keys + 16 * (uint64_t)s->owner, s->nonce, NULL, 0,
-                                tmp, s->len, tmp, tags_out + 16 * i);
+        gift_oracle_gcm_encrypt(keys + 16 * (uint64_t)s->owner, s->nonce, aad16 ? aad16 + 16 * i : NULL,
+                                aad16 ? 16 : 0, tmp, s->len, tmp, tags_out + 16 * i);
         seg_scatter(&e, s, dst, tmp);
         free(tmp);
     }
@@ -519,7 +521,7 @@ int gift_oracle_seg_decrypt(const uint8_t* src, uint8_t* dst, uint64_t buf_bytes
                             const int32_t* page_table, uint32_t n_pages, uint64_t page_bytes,
                             int32_t* owner_map, uint32_t n_units, uint64_t unit_bytes,
                             const uint8_t* keys, const uint8_t* has_key, uint32_t max_users,
-                            const uint8_t* tags_in, uint32_t* status, int mode)
+                            const uint8_t* tags_in, uint32_t* status, int mode, const uint8_t* aad16)
 {
     seg_env e = { src, dst, buf_bytes, page_table, n_pages, page_bytes,
                   owner_map, n_units, unit_bytes, keys, has_key, max_users };
@@ -543,8 +545,8 @@ int gift_oracle_seg_decrypt(const uint8_t* src, uint8_t* dst, uint64_t buf_bytes
         uint8_t* tmp = (uint8_t*)malloc(s->len ? s->len : 1);
         if (!tmp) { failed = 1; continue; }
         seg_gather(&e, s, src, tmp);
-        int bad = gift_oracle_gcm_decrypt(keys + 16 * (uint64_t)s->owner, s->nonce, NULL, 0,
-                                          tmp, s->len, tags_in + 16 * i, tmp);
+        int bad = gift_oracle_gcm_decrypt(keys + 16 * (uint64_t)s->owner, s->nonce, aad16 ? aad16 + 16 * i : NULL,
+                                          aad16 ? 16 : 0, tmp, s->len, tags_in + 16 * i, tmp);
         status[i] = bad ? ST_TAG_MISMATCH : 0;
         if (mode == 0) {
             if (bad) memset(tmp, 0, s->len);

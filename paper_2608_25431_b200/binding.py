@@ -23,7 +23,7 @@ STATIC_MAX_SEGS = 65536
 
 EXPORTS = [
     "gift_ctx_create", "gift_ctx_destroy", "gift_ctx_reserve", "gift_set_keys", "gift_clear_keys",
-    "gift_seg_encrypt", "gift_seg_encrypt_static", "gift_seg_decrypt", "gift_verify_tags",
+    "gift_ctx_bind_aad", "gift_seg_encrypt", "gift_seg_encrypt_static", "gift_seg_decrypt", "gift_verify_tags",
     "gift_propagate_labels", "gift_tok_encrypt", "gift_tok_decrypt", "gift_check_launch_order",
     "gift_resolve_args", "gift_slice_runs", "gift_expand_owners", "gift_labels_swap_out", "gift_labels_swap_in",
     "gift_strerror", "gift_version", "gift_launch_count", "gift_timing_enable", "gift_timing_read",
@@ -216,6 +216,13 @@ class Ctx:
     def __exit__(self, *exc):
         self.close()
 
+    def bind_aad(self, aad16):
+        """aad16: CUDA uint8 tensor [nseg, 16] authenticated with the segments of the calls that follow, or None."""
+        f = lib().gift_ctx_bind_aad
+        f.argtypes = [C.c_void_p, C.c_void_p]
+        self._aad = aad16            # keep the tensor alive while it is bound
+        _check(f(self._h, _dev(aad16)), "gift_ctx_bind_aad")
+
     def reserve(self, max_segs: int):
         _check(lib().gift_ctx_reserve(self._h, max_segs), "gift_ctx_reserve")
 
@@ -367,6 +374,10 @@ def gift_ctx_create(max_users: int, device: int = 0, flags: int = 0) -> Ctx:
 
 def gift_ctx_destroy(ctx: Ctx):
     ctx.close()
+
+
+def gift_ctx_bind_aad(ctx: Ctx, aad16):
+    ctx.bind_aad(aad16)
 
 
 def gift_ctx_reserve(ctx: Ctx, max_segs: int):

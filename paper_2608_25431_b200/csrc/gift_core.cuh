@@ -307,17 +307,26 @@ GIFT_HD u128 run_lane_rows(const Tab& tb, const uint32_t* rk, const CtrPrefix& p
     return mul_by_power(acc, powtab, e);
 }
 
-// Tag from the combined hash S of all runs: T = (S + LEN*H) ^ E_K(J0), as four LE words.
+// Tag from the combined hash S of all runs: T = (S + A*H^(n+2) + LEN*H) ^ E_K(J0), as four LE
+// words.  A is an optional 16-byte block of additional authenticated data (SP 800-38D
+// sec. 7.1: the AAD blocks precede the ciphertext in GHASH); aad == nullptr means none.
 template <class Tab>
 GIFT_HD void finish_tag(const Tab& tb, const uint32_t* rk, const uint32_t h[4], const uint32_t nonce[3],
-                        uint64_t len_bytes, const u128& s, uint32_t tag[4])
+                        uint64_t len_bytes, const u128& s, uint32_t tag[4], const uint8_t* aad = nullptr,
+                        const u128* powtab = nullptr)
 {
-    // length block [0]_64 || [8*len]_64, big-endian bytes, as LE words then natural domain
+    // length block [8*|A|]_64 || [8*|C|]_64, big-endian bytes, as LE words then natural domain
     const uint64_t bits = len_bytes * 8;
-    const u128 lenf = block_to_field(0u, 0u, bswap32((uint32_t)(bits >> 32)), bswap32((uint32_t)bits));
+    const u128 lenf = block_to_field(0u, aad ? bswap32(128u) : 0u, bswap32((uint32_t)(bits >> 32)),
+                                     bswap32((uint32_t)bits));
     u128 hh;
     hh.w[0] = h[0]; hh.w[1] = h[1]; hh.w[2] = h[2]; hh.w[3] = h[3];
-    const u128 t = xor128(s, gfmul(lenf, hh));
+    u128 t = xor128(s, gfmul(lenf, hh));
+    if (aad) {
+        const Block a = load_block(aad);
+        const uint64_t nblk = (len_bytes + 15) >> 4;
+        t = xor128(t, mul_by_power(block_to_field(a.d[0], a.d[1], a.d[2], a.d[3]), powtab, nblk + 2));
+    }
     uint32_t j0[4] = {nonce[0], nonce[1], nonce[2], 0x01000000u};     // nonce || 00 00 00 01
     aes128_encrypt(tb, rk, j0);
     tag[0] = reflect_bytes(t.w[0]) ^ j0[0];

@@ -44,6 +44,7 @@ struct gift_ctx {
     uint32_t order_cap;
     int32_t* d_snapshot;               // label snapshot for aliased rules
     uint32_t snapshot_cap;
+    const uint8_t* aad;                // per-segment additional authenticated data bound to the next calls, or nullptr
     uint64_t launches;
     int timing;                        // record events around the cipher kernel
     uint32_t n_timed;

@@ -236,3 +236,35 @@ def test_key_change_touches_only_that_user_and_clear_keys():
     _, st = gpu_encrypt(ctx, w, c)
     assert st_(st).tolist() == [0, 0, 8, 0, 0, 0, 0, 0]
     ctx.close()
+
+
+def test_bound_aad_matches_oracle_and_detects_a_changed_role():
+    from oracle import gcm
+    for w in (W.config1(), W.config4(total_bytes=6 << 20, cap_bytes=2 << 20, n_users=8)):
+        n = len(w.segs)
+        rng = np.random.default_rng(31)
+        aad = np.frombuffer(rng.bytes(16 * n), dtype=np.uint8).reshape(n, 16).copy()
+        ctx = make_ctx(w)
+        d_aad = dev(aad)
+        ctx.bind_aad(d_aad)
+        buf = dev(w.buf)
+        tags, st = gpu_encrypt(ctx, w, buf)
+        ref = w.buf.copy()
+        ref_tags, ref_st = gcm.seg_encrypt(ref, ref, w.segs, w.user_ids, w.keys, w.max_users, w.page_table,
+                                           w.page_bytes, w.owner_map, w.unit_bytes, aad=aad)
+        assert np.array_equal(st_(st), ref_st) and np.array_equal(np_(tags), ref_tags) and np.array_equal(np_(buf), ref)
+        st = gpu_decrypt(ctx, w, buf, tags, verify_only=True)
+        assert not st_(st).any()
+        moved = aad.copy()
+        moved[n // 2, 5] ^= 0x10
+        ctx.bind_aad(dev(moved))
+        st = gpu_decrypt(ctx, w, buf, tags, verify_only=True)
+        expect = gcm.seg_decrypt(ref, ref.copy(), w.segs, ref_tags, w.user_ids, w.keys, w.max_users, w.page_table,
+                                 w.page_bytes, verify_only=True, aad=moved)
+        assert np.array_equal(st_(st), expect) and expect[n // 2] == 1 and expect.sum() == 1
+        ctx.bind_aad(None)                       # unbound again: plain tags
+        buf2 = dev(w.buf)
+        tags2, _ = gpu_encrypt(ctx, w, buf2)
+        plain_tags, _ = oracle_encrypt(w, w.buf.copy(), w.buf.copy())
+        assert np.array_equal(np_(tags2), plain_tags)
+        ctx.close()

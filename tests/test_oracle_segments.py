@@ -171,3 +171,25 @@ def test_workload_generators_are_seeded():
     w3 = W.config3(layers=1, n_users=2, min_len=17, max_len=40, fill=True)
     assert w3.buf.size == len(w3.segs) * W.KV_PAGE_BYTES
     assert sorted(w3.page_table.tolist()) == list(range(len(w3.segs)))
+
+
+def test_segment_aad_matches_openssl_and_binds_the_tag():
+    w = W.config1()
+    rng = np.random.default_rng(3)
+    aad = np.frombuffer(rng.bytes(16 * len(w.segs)), dtype=np.uint8).reshape(-1, 16)
+    ct = w.buf.copy()
+    tags, st = gcm.seg_encrypt(w.buf, ct, w.segs, w.user_ids, w.keys, w.max_users, aad=aad)
+    assert not st.any()
+    for i, s in enumerate(w.segs):
+        o, n = int(s["offset"]), int(s["len"])
+        ref = AESGCM(w.keys[int(s["owner"])].tobytes()).encrypt(s["nonce"].tobytes(), w.buf[o:o + n].tobytes(),
+                                                                aad[i].tobytes())
+        assert ct[o:o + n].tobytes() + tags[i].tobytes() == ref
+    plain_tags, _ = gcm.seg_encrypt(w.buf, w.buf.copy(), w.segs, w.user_ids, w.keys, w.max_users)
+    assert not np.array_equal(tags, plain_tags)                      # the data is authenticated, not ignored
+    st = gcm.seg_decrypt(ct, ct.copy(), w.segs, tags, w.user_ids, w.keys, w.max_users, aad=aad)
+    assert not st.any()
+    moved = aad.copy()
+    moved[2, 0] ^= 1                                                 # presented in another role
+    st = gcm.seg_decrypt(ct, ct.copy(), w.segs, tags, w.user_ids, w.keys, w.max_users, aad=moved)
+    assert st.tolist() == [0, 0, 1, 0, 0, 0, 0, 0]
