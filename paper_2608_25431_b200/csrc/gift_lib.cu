@@ -94,6 +94,7 @@ struct CallArgs {
     uint32_t n_units;
     uint64_t unit_bytes;
     uint8_t* tags;                 // out (encrypt) or in (decrypt, verify)
+    const uint8_t* aad;            // 16 bytes of additional authenticated data per segment, or nullptr
     uint32_t* status;
     const KeyHot* hot;
     const u128* pow;
@@ -425,7 +426,8 @@ __global__ void __launch_bounds__(THREADS, 1) crypt_kernel(CallArgs a, const uin
         }
         if (last) {
             uint32_t tag[4];
-            finish_tag(tb, rk, slot->h, nonce, seg.len, sum, tag);
+            finish_tag(tb, rk, slot->h, nonce, seg.len, sum, tag, a.aad ? a.aad + 16 * (size_t)s : nullptr,
+                       a.pow + (size_t)seg.owner * (POW_LEVELS * 256));
             uint4* tagp = reinterpret_cast<uint4*>(a.tags) + s;
             if (MODE == MODE_ENCRYPT) {
                 if (lane == 0) *tagp = make_uint4(tag[0], tag[1], tag[2], tag[3]);
@@ -687,6 +689,7 @@ int seg_call(gift_ctx* c, const void* src, void* dst, uint64_t buf_bytes, const 
     if (pages) { a.page_table = pages->table; a.n_pages = pages->n; a.page_bytes = pages->page_bytes; }
     if (labels) { a.owner_map = labels->owner_map; a.n_units = labels->n_units; a.unit_bytes = labels->unit_bytes; }
     a.tags = tags;
+    a.aad = c->aad;
     a.status = status;
     a.hot = c->d_hot;
     a.pow = c->d_pow;
@@ -953,6 +956,14 @@ int gift_propagate_labels(gift_ctx* c, const gift_rule* rule, const int32_t* con
         c->launches++;
     }
     CU_TRY(cudaGetLastError());
+    return GIFT_OK;
+}
+
+int gift_ctx_bind_aad(gift_ctx* c, const uint8_t* aad16)
+{
+    if (!c) return GIFT_E_INVAL;
+    if ((uintptr_t)aad16 & 15) return GIFT_E_ALIGN;
+    c->aad = aad16;
     return GIFT_OK;
 }
 
