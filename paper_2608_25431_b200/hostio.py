@@ -110,3 +110,53 @@ class HostExporter:
         for st in self.streams:
             cur.wait_stream(st)
 
+
+class StepPipeline:
+    """Whole-buffer export steps kept two in flight: for tables whose segments cannot be cut
+    into contiguous chunks (page chains scattered over the pool).  Step i runs upload, export
+    and download on stream i mod 2 with its own context and device buffers, so the download
+    of one step overlaps the upload of the next."""
+
+    def __init__(self, max_users: int, user_ids, keys, buf_bytes: int, nseg: int, device: int = 0, flags: int = 0):
+        self.ctxs = [binding.Ctx(max_users, device, flags) for _ in range(2)]
+        for c in self.ctxs:
+            c.set_keys(user_ids, keys)
+            c.reserve(nseg)
+        self.streams = [torch.cuda.Stream(device=device) for _ in range(2)]
+        dev = torch.device("cuda", device)
+        self.bufs = [torch.empty(buf_bytes, dtype=torch.uint8, device=dev) for _ in range(2)]
+        self.tags = [torch.empty((nseg, 16), dtype=torch.uint8, device=dev) for _ in range(2)]
+        self.status = [torch.empty(nseg, dtype=torch.int32, device=dev) for _ in range(2)]
+        self.h_out = [torch.empty(buf_bytes, dtype=torch.uint8, pin_memory=True) for _ in range(2)]
+        self.h_tags = [torch.empty((nseg, 16), dtype=torch.uint8, pin_memory=True) for _ in range(2)]
+        self.h_status = [torch.empty(nseg, dtype=torch.int32, pin_memory=True) for _ in range(2)]
+        self.step_no = 0
+
+    def close(self):
+        for c in self.ctxs:
+            c.close()
+
+    def launch_count(self) -> int:
+        return sum(c.launch_count() for c in self.ctxs)
+
+    def step(self, h_src: torch.Tensor, d_segs: torch.Tensor, nseg: int, page_table=None, page_bytes: int = 0,
+             owner_map=None, unit_bytes: int = 0):
+        """Enqueue one export step; returns the slot (0/1) whose host outputs it will fill."""
+        k = self.step_no & 1
+        self.step_no += 1
+        st = self.streams[k]
+        st.wait_stream(torch.cuda.current_stream())
+        with torch.cuda.stream(st):
+            self.bufs[k].copy_(h_src, non_blocking=True)
+            self.ctxs[k].seg_encrypt(self.bufs[k], self.bufs[k], d_segs, nseg, self.tags[k], self.status[k],
+                                     page_table=page_table, page_bytes=page_bytes, owner_map=owner_map,
+                                     unit_bytes=unit_bytes, stream=st.cuda_stream)
+            self.h_out[k].copy_(self.bufs[k], non_blocking=True)
+            self.h_tags[k].copy_(self.tags[k], non_blocking=True)
+            self.h_status[k].copy_(self.status[k], non_blocking=True)
+        return k
+
+    def wait(self):
+        for st in self.streams:
+            torch.cuda.current_stream().wait_stream(st)
+

@@ -61,3 +61,34 @@ def test_layer_chunked_export_matches_oracle():
     assert np.array_equal(h_status.numpy().astype(np.uint32), st_ref)
     assert np.array_equal(d_buf.cpu().numpy(), pt_ref) and np.array_equal(om_dev.cpu().numpy(), om_ref)
     exp.close()
+
+
+def test_two_steps_in_flight_match_oracle():
+    w = W.config4(total_bytes=6 << 20, cap_bytes=2 << 20, n_users=8)
+    nseg = len(w.segs)
+    pipe = hostio.StepPipeline(w.max_users, w.user_ids, w.keys, w.buf_bytes, nseg)
+    d_segs = torch.from_numpy(w.segs.view(np.uint8).copy()).cuda()
+    table, om = torch.from_numpy(w.page_table).cuda(), torch.from_numpy(w.owner_map).cuda()
+    rng = np.random.default_rng(8)
+    inputs = [torch.from_numpy(np.frombuffer(rng.bytes(w.buf_bytes), dtype=np.uint8).copy()).pin_memory()
+              for _ in range(3)]
+    slots = []
+    for h in inputs[:2]:                                     # two steps in flight at once
+        slots.append(pipe.step(h, d_segs, nseg, page_table=table, page_bytes=w.page_bytes, owner_map=om,
+                               unit_bytes=w.unit_bytes))
+    pipe.wait()
+    torch.cuda.synchronize()
+    assert slots == [0, 1]
+    for h, k in zip(inputs[:2], slots):
+        ref = h.numpy().copy()
+        ref_tags, ref_st = oracle_encrypt(w, ref, ref)
+        assert np.array_equal(pipe.h_out[k].numpy(), ref) and np.array_equal(pipe.h_tags[k].numpy(), ref_tags)
+        assert np.array_equal(pipe.h_status[k].numpy().astype(np.uint32), ref_st)
+    k = pipe.step(inputs[2], d_segs, nseg, page_table=table, page_bytes=w.page_bytes, owner_map=om,
+                  unit_bytes=w.unit_bytes)                   # slot 0 again
+    pipe.wait()
+    torch.cuda.synchronize()
+    ref = inputs[2].numpy().copy()
+    ref_tags, _ = oracle_encrypt(w, ref, ref)
+    assert k == 0 and np.array_equal(pipe.h_out[0].numpy(), ref) and np.array_equal(pipe.h_tags[0].numpy(), ref_tags)
+    pipe.close()
