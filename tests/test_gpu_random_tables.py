@@ -84,3 +84,30 @@ def test_random_tables_match_oracle(paged, page_bytes):
         assert np.array_equal(st_(st2), st_ref), (paged, page_bytes, trial)
         assert np.array_equal(np_(d_bad), out_ref) and np.array_equal(np_(om), om_ref)
         ctx.close()
+
+
+def test_many_tiny_segments():
+    """200 000 segments of 0..80 bytes: one run each; stresses the work list, the scan and the scratch growth."""
+    rng = np.random.default_rng(W.SEED_BASE + 90)
+    nseg, n_users = 200_000, 64
+    lens = rng.integers(0, 81, size=nseg)
+    offs = np.arange(nseg, dtype=np.uint64) * np.uint64(96)
+    segs = np.zeros(nseg, dtype=W.SEG_DTYPE)
+    segs["owner"] = rng.integers(0, n_users, size=nseg)
+    segs["offset"] = offs
+    segs["len"] = lens
+    segs["nonce"][:, :4] = np.arange(nseg, dtype="<u4")[:, None].view(np.uint8).reshape(nseg, 4)
+    ids = np.arange(n_users, dtype=np.int32)
+    keys = np.frombuffer(rng.bytes(16 * n_users), dtype=np.uint8).reshape(n_users, 16).copy()
+    buf = np.frombuffer(rng.bytes(nseg * 96), dtype=np.uint8).copy()
+    w = W.Workload("tiny", ids, keys, n_users, buf, buf.size, segs)
+    ctx = make_ctx(w)
+    d = dev(buf)
+    tags, st = gpu_encrypt(ctx, w, d)
+    ref = buf.copy()
+    ref_tags, ref_st = gcm.seg_encrypt(ref, ref, segs, ids, keys, n_users)
+    assert not ref_st.any() and np.array_equal(st_(st), ref_st)
+    assert np.array_equal(np_(tags), ref_tags) and np.array_equal(np_(d), ref)
+    st2 = gpu_decrypt(ctx, w, d, tags)
+    assert not st_(st2).any() and np.array_equal(np_(d), buf)
+    ctx.close()
