@@ -6,8 +6,9 @@ python bench.py --impl reference --steps K --warmup W    # the CPU oracle, timed
 Workload (default): the prefill -> decode KV-cache handoff of a LLaMA-7B-shaped model
 (workloads.config3 at 32 layers): every 256 KiB KV block of every user encrypted under its
 owner's key with a per-block tag.  One step = one pass of the whole hot path over that
-batch: the flow rule of the handoff copy on the block owner map (IDENTITY), then
-gift_seg_encrypt (plan + label check, work list, CTR + GHASH, tag finish) in place.  Key
+batch: the four flow rules on the blocks' owner labels (copy, row-preserving, per-group
+reduction, scatter to pool pages), then gift_seg_encrypt (plan + label check, work list,
+CTR + GHASH, tag finish) in place.  Key
 setup is outside the step, as it is once per key change.  The path does not shard: with
 --gpus N every rank runs an independent replica on its own GPU (no collective on the data
 path) and the value is the sum of the replicas over the slowest rank's time.
@@ -257,10 +258,37 @@ def main():
     flush = torch.empty(512 << 20, dtype=torch.uint8, device="cuda") if w.payload_bytes <= (256 << 20) else None
     payload = w.payload_bytes
 
+    # Flow rules of the step.  For the KV handoff the labels start per segment in table order
+    # (layer-major, each user's blocks contiguous) and pass through all four rule kinds: the
+    # copy (IDENTITY), a row-preserving kernel with a parameter operand (ROWWISE), a reduction
+    # per (layer, user) over that group's blocks (SEGREDUCE) and the scatter to physical pool
+    # pages through the inverse block table (BROADCAST).  The result is the page owner map that
+    # the export's label check reads.  Other workloads apply the copy rule to their unit map.
+    rules4 = None
+    if args.workload == "c3":
+        x = w.extra
+        om_seg = torch.from_numpy(w.segs["owner"].astype(np.int32)).cuda()
+        tmp_a, tmp_b = torch.empty_like(om_seg), torch.empty_like(om_seg)
+        param = torch.full((1,), binding.OWNER_PARAM, dtype=torch.int32, device="cuda")
+        grp = np.concatenate([[0], np.cumsum(np.tile(x["nblk"], x["layers"]))]).astype(np.int32)
+        grp_ptr = torch.from_numpy(grp).cuda()
+        src_idx = torch.arange(nseg, dtype=torch.int32, device="cuda")
+        inv = np.empty(nseg, dtype=np.int32)
+        inv[w.page_table] = np.arange(nseg, dtype=np.int32)
+        inv_table = torch.from_numpy(inv).cuda()
+        rules4 = (om_seg, tmp_a, tmp_b, param, grp_ptr, src_idx, inv_table)
+
     def step():
         if flush is not None:
             flush.fill_(1)
-        ctx.propagate_labels(binding.RULE_IDENTITY, [om_src], om, viol)
+        if rules4 is not None:
+            ctx.propagate_labels(binding.RULE_IDENTITY, [om_seg], tmp_a, viol)
+            ctx.propagate_labels(binding.RULE_ROWWISE, [tmp_a, param], tmp_b, viol, param_mask=2)
+            ctx.propagate_labels(binding.RULE_SEGREDUCE, [tmp_b, tmp_b], tmp_a, viol, seg_ptr=grp_ptr, src_ptr=grp_ptr,
+                                 src_idx=src_idx)
+            ctx.propagate_labels(binding.RULE_BROADCAST, [tmp_a], om, viol, gather=inv_table)
+        else:
+            ctx.propagate_labels(binding.RULE_IDENTITY, [om_src], om, viol)
         ctx.seg_encrypt(buf, buf, segs, nseg, tags, status, page_table=table, page_bytes=w.page_bytes,
                         owner_map=om, unit_bytes=w.unit_bytes)
 
@@ -268,6 +296,7 @@ def main():
         step()
     barrier()
     assert not status.any().item() and int(viol[0].item()) == 0, "workload segments were rejected"
+    assert torch.equal(om, om_src), "propagated labels differ from the pool's owner map"
     l0 = ctx.launch_count()
     ctx.timing_enable(True)
     sampler = ClockSampler(physical_gpu_index(local))
