@@ -140,7 +140,10 @@ int gift_clear_keys(gift_ctx* ctx, const int32_t* user_ids, uint32_t n, void* st
  * 16-byte GCM tag.  Otherwise the segment's dst bytes are left as they were,
  * its tag is 16 zero bytes and status[i] says why.  src may equal dst; bytes
  * outside all segments are never written.  Segments of one call must not
- * overlap.  buf_bytes is the size of src and of dst. */
+ * overlap.  buf_bytes is the size of src and of dst.  src and dst are addresses
+ * the device can dereference: device memory, or page-locked host memory mapped
+ * into the device's address space (the boundary copy of sec. 4.5 fused into
+ * the cipher: the kernel then reads or writes across the bus itself). */
 int gift_seg_encrypt(gift_ctx* ctx, const void* src, void* dst, uint64_t buf_bytes,
                      const gift_seg* segs, uint32_t nseg, const gift_pages* pages,
                      const gift_labels* labels, uint8_t* tags_out, uint32_t* status, void* stream);

@@ -179,11 +179,12 @@ def _stream_ptr(stream):
 
 
 def _dev(t):
-    """Device pointer of a CUDA tensor (or None)."""
+    """Device-visible pointer of a contiguous CUDA tensor, or of a pinned host tensor (page-locked
+    host memory has the same address on the device under unified addressing), or None."""
     if t is None:
         return None
-    if not t.is_cuda or not t.is_contiguous():
-        raise ValueError("expected a contiguous CUDA tensor")
+    if not (t.is_cuda or t.is_pinned()) or not t.is_contiguous():
+        raise ValueError("expected a contiguous CUDA tensor or a pinned host tensor")
     return C.c_void_p(t.data_ptr())
 
 

@@ -60,11 +60,13 @@ class HostExporter:
     def export(self, h_src: torch.Tensor, h_dst: torch.Tensor, d_buf: torch.Tensor, chunks: List[Chunk],
                d_segs: torch.Tensor, d_tags: torch.Tensor, d_status: torch.Tensor, h_tags: torch.Tensor,
                h_status: torch.Tensor, page_table: Optional[torch.Tensor] = None, page_bytes: int = 0,
-               owner_map: Optional[torch.Tensor] = None, unit_bytes: int = 0):
+               owner_map: Optional[torch.Tensor] = None, unit_bytes: int = 0, direct_out: bool = False):
         """Enqueue upload, export and download of every chunk; returns without waiting.
 
         h_src, h_dst: pinned uint8 host tensors of the buffer's size; d_buf: device staging of
-        the same size; d_segs: the whole table on the device as uint8[nseg*40].
+        the same size; d_segs: the whole table on the device as uint8[nseg*40].  With
+        direct_out the cipher kernel stores the ciphertext straight into h_dst (pinned memory is
+        device-visible), so the staged plaintext stays intact and no download copy runs.
         """
         cur = torch.cuda.current_stream()
         start = torch.cuda.Event()
@@ -76,11 +78,12 @@ class HostExporter:
             with torch.cuda.stream(st):
                 d_buf[ch.byte_lo:ch.byte_hi].copy_(h_src[ch.byte_lo:ch.byte_hi], non_blocking=True)
                 n = ch.seg_hi - ch.seg_lo
-                ctx.seg_encrypt(d_buf, d_buf, d_segs[ch.seg_lo * 40: ch.seg_hi * 40], n,
+                ctx.seg_encrypt(d_buf, h_dst if direct_out else d_buf, d_segs[ch.seg_lo * 40: ch.seg_hi * 40], n,
                                 d_tags[ch.seg_lo:ch.seg_hi], d_status[ch.seg_lo:ch.seg_hi],
                                 page_table=page_table, page_bytes=page_bytes, owner_map=owner_map,
                                 unit_bytes=unit_bytes, stream=st.cuda_stream)
-                h_dst[ch.byte_lo:ch.byte_hi].copy_(d_buf[ch.byte_lo:ch.byte_hi], non_blocking=True)
+                if not direct_out:
+                    h_dst[ch.byte_lo:ch.byte_hi].copy_(d_buf[ch.byte_lo:ch.byte_hi], non_blocking=True)
                 h_tags[ch.seg_lo:ch.seg_hi].copy_(d_tags[ch.seg_lo:ch.seg_hi], non_blocking=True)
                 h_status[ch.seg_lo:ch.seg_hi].copy_(d_status[ch.seg_lo:ch.seg_hi], non_blocking=True)
         for st in self.streams:

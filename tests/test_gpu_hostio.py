@@ -92,3 +92,30 @@ def test_two_steps_in_flight_match_oracle():
     ref_tags, _ = oracle_encrypt(w, ref, ref)
     assert k == 0 and np.array_equal(pipe.h_out[0].numpy(), ref) and np.array_equal(pipe.h_tags[0].numpy(), ref_tags)
     pipe.close()
+
+
+def test_direct_output_into_pinned_host_memory_matches_oracle():
+    """The cipher kernel stores ciphertext straight into pinned host memory; the staged plaintext stays."""
+    w = W.config3(layers=3, n_users=5, min_len=40, max_len=300)
+    nseg, n_slots = len(w.segs), w.extra["n_slots"]
+    ref = w.buf.copy()
+    ref_tags, ref_st = oracle_encrypt(w, ref, ref)
+    assert not ref_st.any()
+    h_src = torch.from_numpy(w.buf).pin_memory()
+    h_dst = torch.zeros(w.buf_bytes, dtype=torch.uint8).pin_memory()
+    h_tags = torch.zeros((nseg, 16), dtype=torch.uint8).pin_memory()
+    h_status = torch.full((nseg,), 9, dtype=torch.int32).pin_memory()
+    d_buf = torch.zeros(w.buf_bytes, dtype=torch.uint8, device="cuda")
+    d_segs = torch.from_numpy(w.segs.view(np.uint8).copy()).cuda()
+    d_tags = torch.zeros((nseg, 16), dtype=torch.uint8, device="cuda")
+    d_status = torch.zeros(nseg, dtype=torch.int32, device="cuda")
+    exp = hostio.HostExporter(w.max_users, w.user_ids, w.keys, 0, 2, 0, n_slots)
+    chunks = hostio.layer_chunks(3, n_slots, n_slots * w.page_bytes)
+    exp.export(h_src, h_dst, d_buf, chunks, d_segs, d_tags, d_status, h_tags, h_status,
+               page_table=torch.from_numpy(w.page_table).cuda(), page_bytes=w.page_bytes, direct_out=True)
+    torch.cuda.synchronize()
+    assert not h_status.any().item()
+    assert np.array_equal(h_tags.numpy(), ref_tags)
+    assert np.array_equal(h_dst.numpy(), ref)
+    assert np.array_equal(d_buf.cpu().numpy(), w.buf)         # the device copy is still plaintext
+    exp.close()
