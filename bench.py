@@ -7,7 +7,7 @@ Workload (default): the prefill -> decode KV-cache handoff of a LLaMA-7B-shaped 
 (workloads.config3 at 32 layers): every 256 KiB KV block of every user encrypted under its
 owner's key with a per-block tag.  One step = one pass of the whole hot path over that
 batch: the four flow rules on the blocks' owner labels (copy, row-preserving, per-group
-reduction, scatter to pool pages), then gift_seg_encrypt (plan + label check, work list,
+reduction, scatter to pool pages; one fused launch), then gift_seg_encrypt (plan + label check, work list,
 CTR + GHASH, tag finish) in place.  Key
 setup is outside the step, as it is once per key change.  The path does not shard: with
 --gpus N every rank runs an independent replica on its own GPU (no collective on the data
@@ -276,17 +276,22 @@ def main():
         inv = np.empty(nseg, dtype=np.int32)
         inv[w.page_table] = np.arange(nseg, dtype=np.int32)
         inv_table = torch.from_numpy(inv).cuda()
-        rules4 = (om_seg, tmp_a, tmp_b, param, grp_ptr, src_idx, inv_table)
+        tmp_c = torch.empty_like(om_seg)
+        rules4 = [
+            {"kind": binding.RULE_IDENTITY, "in_maps": [om_seg], "out_map": tmp_a},
+            {"kind": binding.RULE_ROWWISE, "in_maps": [tmp_a, param], "out_map": tmp_b, "param_mask": 2},
+            {"kind": binding.RULE_SEGREDUCE, "in_maps": [tmp_b, tmp_b], "out_map": tmp_c, "seg_ptr": grp_ptr,
+             "src_ptr": grp_ptr, "src_idx": src_idx},
+            {"kind": binding.RULE_BROADCAST, "in_maps": [tmp_c], "out_map": om, "gather": inv_table},
+        ]
+        viol4 = torch.zeros(8, dtype=torch.int32, device="cuda")
+        run_rules4 = ctx.prepare_chain(rules4)
 
     def step():
         if flush is not None:
             flush.fill_(1)
         if rules4 is not None:
-            ctx.propagate_labels(binding.RULE_IDENTITY, [om_seg], tmp_a, viol)
-            ctx.propagate_labels(binding.RULE_ROWWISE, [tmp_a, param], tmp_b, viol, param_mask=2)
-            ctx.propagate_labels(binding.RULE_SEGREDUCE, [tmp_b, tmp_b], tmp_a, viol, seg_ptr=grp_ptr, src_ptr=grp_ptr,
-                                 src_idx=src_idx)
-            ctx.propagate_labels(binding.RULE_BROADCAST, [tmp_a], om, viol, gather=inv_table)
+            run_rules4(viol4)                           # the four rules in one launch
         else:
             ctx.propagate_labels(binding.RULE_IDENTITY, [om_src], om, viol)
         ctx.seg_encrypt(buf, buf, segs, nseg, tags, status, page_table=table, page_bytes=w.page_bytes,
@@ -297,6 +302,7 @@ def main():
     barrier()
     assert not status.any().item() and int(viol[0].item()) == 0, "workload segments were rejected"
     assert torch.equal(om, om_src), "propagated labels differ from the pool's owner map"
+    assert rules4 is None or not viol4[0::2].any().item(), "a flow rule reported a conflict"
     l0 = ctx.launch_count()
     ctx.timing_enable(True)
     sampler = ClockSampler(physical_gpu_index(local))
@@ -421,6 +427,41 @@ def main():
                                                                gather=ga5), n=50) * 1e3,
             "tokens": int(t_own.numel()), "violations_last": int(viol[0].item()),
         }
+        ta, tb, tc = torch.empty_like(t_own), torch.empty_like(t_own), torch.empty_like(t_own)
+        chain5 = [
+            {"kind": binding.RULE_IDENTITY, "in_maps": [t_own], "out_map": ta},
+            {"kind": binding.RULE_ROWWISE, "in_maps": [ta, par], "out_map": tb, "param_mask": 2},
+            {"kind": binding.RULE_SEGREDUCE, "in_maps": [tb, kv_own], "out_map": tc, "seg_ptr": sp5, "src_ptr": srcp5,
+             "src_idx": bt5},
+            {"kind": binding.RULE_BROADCAST, "in_maps": [tc], "out_map": t_out, "gather": ga5},
+        ]
+        v8 = torch.zeros(8, dtype=torch.int32, device="cuda")
+        run_chain5 = ctx.prepare_chain(chain5)
+        rules["fused_chain_of_4_us"] = timed(lambda: run_chain5(v8), n=50) * 1e3
+        rules["fused_chain_ok"] = bool(torch.equal(t_out, t_own) and not v8[0::2].any().item())
+
+        # the direct numbers above include this binding's per-call marshalling on the host; replayed
+        # CUDA graphs of the same launches give the device side alone
+        def four_separate():
+            ctx.propagate_labels(binding.RULE_IDENTITY, [t_own], ta, viol)
+            ctx.propagate_labels(binding.RULE_ROWWISE, [ta, par], tb, viol, param_mask=2)
+            ctx.propagate_labels(binding.RULE_SEGREDUCE, [tb, kv_own], tc, viol, seg_ptr=sp5, src_ptr=srcp5, src_idx=bt5)
+            ctx.propagate_labels(binding.RULE_BROADCAST, [tc], t_out, viol, gather=ga5)
+
+        def graph_us(fn):
+            side = torch.cuda.Stream()
+            side.wait_stream(torch.cuda.current_stream())
+            with torch.cuda.stream(side):
+                fn()
+            torch.cuda.current_stream().wait_stream(side)
+            torch.cuda.synchronize()
+            g = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(g):
+                fn()
+            return timed(g.replay, n=50) * 1e3
+
+        rules["four_separate_rules_graph_us"] = graph_us(four_separate)
+        rules["fused_chain_of_4_graph_us"] = graph_us(lambda: run_chain5(v8))
         # a decode step's output rows (config 2: 256 rows of 64 004 B): direct calls and a replayed CUDA graph
         w2 = W.config2()
         c2 = binding.Ctx(w2.max_users, local, args.flags)

@@ -267,6 +267,22 @@ typedef struct {
 int gift_propagate_labels(gift_ctx* ctx, const gift_rule* rule, const int32_t* const* in_owner_maps,
                           int32_t* out_owner_map, uint32_t* viol, void* stream);
 
+/* The rules of consecutive kernels applied in one launch (paper sec. 4.3 runs the rule of
+ * every kernel of a forward pass; a label map is a few hundred KiB, so a rule on its own
+ * costs only its launch).  Rule k is rules[k] with inputs in_owner_maps[k] (HOST array of
+ * its n_in device pointers) and output out_owner_maps[k]; it sees everything rules 0..k-1
+ * wrote, exactly as n_rules calls of gift_propagate_labels in that order would.  viol is a
+ * device array of 2*n_rules words: viol[2k] the number of CONFLICT outputs of rule k and
+ * viol[2k+1] the smallest such index (0xFFFFFFFF if none).  n_rules <= GIFT_CHAIN_MAX, else
+ * GIFT_E_RANGE.  Unlike gift_propagate_labels the chain takes no snapshot: a rule's output
+ * must not overlap the map it gathers from (BROADCAST in0, SEGREDUCE in1), else
+ * GIFT_E_INVAL; writing a map in place at the same index (IDENTITY, ROWWISE, SEGREDUCE
+ * in0) is fine.  One launch of a single 8-CTA cluster: meant for maps of up to a few
+ * million units. */
+#define GIFT_CHAIN_MAX 8u
+int gift_propagate_chain(gift_ctx* ctx, const gift_rule* rules, const int32_t* const* const* in_owner_maps,
+                         int32_t* const* out_owner_maps, uint32_t n_rules, uint32_t* viol, void* stream);
+
 /* Multi-stream launch-order check (paper sec. 4.4, "Concurrency control"): the ownership
  * record of a segment is extended with its last writer kernel and last reader kernels, each
  * a (stream, sequence) pair, and a kernel counts as completed once a synchronisation of its

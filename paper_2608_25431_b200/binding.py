@@ -24,7 +24,7 @@ STATIC_MAX_SEGS = 65536
 EXPORTS = [
     "gift_ctx_create", "gift_ctx_destroy", "gift_ctx_reserve", "gift_set_keys", "gift_clear_keys",
     "gift_ctx_bind_aad", "gift_seg_encrypt", "gift_seg_encrypt_static", "gift_seg_decrypt", "gift_verify_tags",
-    "gift_propagate_labels", "gift_tok_encrypt", "gift_tok_decrypt", "gift_check_launch_order",
+    "gift_propagate_labels", "gift_propagate_chain", "gift_tok_encrypt", "gift_tok_decrypt", "gift_check_launch_order",
     "gift_resolve_args", "gift_slice_runs", "gift_expand_owners", "gift_labels_swap_out", "gift_labels_swap_in",
     "gift_strerror", "gift_version", "gift_launch_count", "gift_timing_enable", "gift_timing_read",
     "gift_probe_pipe",
@@ -141,6 +141,8 @@ def lib():
                                        C.POINTER(_Pages), C.c_void_p, C.c_void_p, C.c_void_p]
         l.gift_propagate_labels.argtypes = [C.c_void_p, C.POINTER(_Rule), C.POINTER(C.c_void_p), C.c_void_p,
                                             C.c_void_p, C.c_void_p]
+        l.gift_propagate_chain.argtypes = [C.c_void_p, C.POINTER(_Rule), C.POINTER(C.POINTER(C.c_void_p)),
+                                           C.POINTER(C.c_void_p), C.c_uint32, C.c_void_p, C.c_void_p]
         l.gift_tok_encrypt.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_uint32, C.c_uint64,
                                        C.c_void_p, C.c_void_p, C.c_void_p]
         l.gift_tok_decrypt.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_uint32, C.c_uint64, C.c_void_p,
@@ -296,6 +298,41 @@ class Ctx:
         _check(lib().gift_propagate_labels(self._h, C.byref(rule), arr, _dev(out_map), _dev(viol),
                                            _stream_ptr(stream)), "gift_propagate_labels")
 
+    def prepare_chain(self, rules):
+        """Marshal a rule chain once; the returned callable (viol, stream=None) runs
+        gift_propagate_chain on it.  `rules` is a list of dicts with the keyword arguments of
+        propagate_labels (kind, in_maps, out_map and the rule's index arrays).  The tensors
+        named in `rules` must stay alive and in place while the callable is used."""
+        n = len(rules)
+        arr = (_Rule * max(n, 1))()
+        ins = (C.POINTER(C.c_void_p) * max(n, 1))()
+        outs = (C.c_void_p * max(n, 1))()
+        keep = [rules]
+        for k, r in enumerate(rules):
+            in_maps, out_map = r["in_maps"], r["out_map"]
+            seg_ptr, src_ptr = r.get("seg_ptr"), r.get("src_ptr")
+            src_idx, gather = r.get("src_idx"), r.get("gather")
+            n_out = r.get("n_out", out_map.numel())
+            arr[k] = _Rule(r["kind"], n_out, len(in_maps), seg_ptr.numel() - 1 if seg_ptr is not None else 0,
+                           in_maps[0].numel(), in_maps[1].numel() if len(in_maps) > 1 else 0,
+                           seg_ptr.data_ptr() if seg_ptr is not None else None,
+                           src_ptr.data_ptr() if src_ptr is not None else None,
+                           src_idx.data_ptr() if src_idx is not None else None,
+                           gather.data_ptr() if gather is not None else None, r.get("param_mask", 0))
+            a = (C.c_void_p * len(in_maps))(*[m.data_ptr() for m in in_maps])
+            keep.append(a)
+            ins[k] = C.cast(a, C.POINTER(C.c_void_p))
+            outs[k] = out_map.data_ptr()
+        fn, h = lib().gift_propagate_chain, self._h
+
+        def run(viol, stream=None, _keep=keep):
+            _check(fn(h, arr, ins, outs, n, _dev(viol), _stream_ptr(stream)), "gift_propagate_chain")
+        return run
+
+    def propagate_chain(self, rules, viol, stream=None):
+        """gift_propagate_chain on `rules` (see prepare_chain); viol holds 2 * len(rules) words."""
+        self.prepare_chain(rules)(viol, stream)
+
     def tok_encrypt(self, tokens, nonces, owners, eos_token, out16, status, stream=None):
         _check(lib().gift_tok_encrypt(self._h, _dev(tokens), _dev(nonces), _dev(owners), tokens.numel(),
                                       int(eos_token), _dev(out16), _dev(status), _stream_ptr(stream)),
@@ -411,6 +448,10 @@ def gift_verify_tags(ctx: Ctx, *args, **kw):
 
 def gift_propagate_labels(ctx: Ctx, *args, **kw):
     ctx.propagate_labels(*args, **kw)
+
+
+def gift_propagate_chain(ctx: Ctx, *args, **kw):
+    ctx.propagate_chain(*args, **kw)
 
 
 def gift_tok_encrypt(ctx: Ctx, *args, **kw):

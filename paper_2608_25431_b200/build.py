@@ -6,8 +6,8 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libgift.so")
 HOSTCHECK = os.path.join(HERE, "libgift_hostcheck.so")
-SOURCES = ["gift_lib.cu", "gift_tokens.cu", "gift_order.cu", "gift_index.cu", "pipe_probe.cu"]
-HEADERS = ["gf128.cuh", "aes_tt.cuh", "gift_core.cuh", "gift_internal.cuh", os.path.join("..", "..", "include", "gift.h")]
+SOURCES = ["gift_lib.cu", "gift_tokens.cu", "gift_order.cu", "gift_index.cu", "gift_chain.cu", "pipe_probe.cu"]
+HEADERS = ["gf128.cuh", "aes_tt.cuh", "gift_core.cuh", "gift_internal.cuh", "gift_rules.cuh", os.path.join("..", "..", "include", "gift.h")]
 
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
               "-shared", "-Xcompiler", "-fPIC"]

@@ -31,6 +31,7 @@ using namespace gift;
 #define GIFT_VERSION 100u   // 0.1.0
 
 #include "gift_internal.cuh"
+#include "gift_rules.cuh"
 
 namespace {
 
@@ -487,48 +488,6 @@ __global__ void fixup_kernel(CallArgs a)
 // label propagation (paper sec. 4.3, rule steps 4 and 5)
 // ---------------------------------------------------------------------------
 
-struct RuleArgs {
-    uint32_t kind, n_out, n_in, n_seg, n_in0, n_in1, param_mask;
-    const int32_t* in[8];
-    const int32_t* seg_ptr;
-    const int32_t* src_ptr;
-    const int32_t* src_idx;
-    const int32_t* gather;
-    int32_t* out;
-    uint32_t* viol;
-};
-
-// The join over a set of labels is decided by three facts: was any label NONE or
-// CONFLICT, the smallest user id seen and the largest one (PARAM is neutral).
-struct JoinAcc {
-    bool bad;
-    int32_t lo, hi;
-    __device__ __forceinline__ void init() { bad = false; lo = 0x7FFFFFFF; hi = -1; }
-    __device__ __forceinline__ void add(int32_t l)
-    {
-        if (l <= GIFT_OWNER_NONE) bad = true;
-        else if (l >= 0) { lo = min(lo, l); hi = max(hi, l); }
-    }
-    __device__ __forceinline__ int32_t result() const
-    {
-        if (bad) return GIFT_OWNER_CONFLICT;
-        if (hi < 0) return GIFT_OWNER_PARAM;
-        return lo == hi ? lo : GIFT_OWNER_CONFLICT;
-    }
-};
-
-__device__ __forceinline__ void report_violation(uint32_t* viol, bool conflict, uint32_t j)
-{
-    const uint32_t m = __ballot_sync(__activemask(), conflict);
-    if (conflict) {
-        const int leader = __ffs(m) - 1;
-        if ((int)(threadIdx.x & 31) == leader) {
-            atomicAdd(viol, (uint32_t)__popc(m));
-            atomicMin(viol + 1, j);      // the leader holds the smallest index of its warp
-        }
-    }
-}
-
 __global__ void rule_pointwise_kernel(RuleArgs r)
 {
     const uint32_t j = blockIdx.x * blockDim.x + threadIdx.x;
@@ -719,12 +678,6 @@ int seg_call(gift_ctx* c, const void* src, void* dst, uint64_t buf_bytes, const 
     return GIFT_OK;
 }
 
-bool ranges_overlap(const void* a, size_t na, const void* b, size_t nb)
-{
-    const uintptr_t a0 = (uintptr_t)a, b0 = (uintptr_t)b;
-    return a0 < b0 + nb && b0 < a0 + na;
-}
-
 }  // namespace
 
 // ---------------------------------------------------------------------------
@@ -897,33 +850,10 @@ int gift_verify_tags(gift_ctx* c, const void* src, uint64_t buf_bytes, const gif
 int gift_propagate_labels(gift_ctx* c, const gift_rule* rule, const int32_t* const* in_maps, int32_t* out,
                           uint32_t* viol, void* stream)
 {
-    if (!c || !rule || !in_maps || !viol) return GIFT_E_INVAL;
-    if (rule->n_out && !out) return GIFT_E_INVAL;
+    if (!c) return GIFT_E_INVAL;
     RuleArgs r;
-    memset(&r, 0, sizeof(r));
-    r.kind = rule->kind; r.n_out = rule->n_out; r.n_in = rule->n_in; r.n_seg = rule->n_seg;
-    r.n_in0 = rule->n_in0; r.n_in1 = rule->n_in1; r.param_mask = rule->param_mask;
-    r.seg_ptr = rule->seg_ptr; r.src_ptr = rule->src_ptr; r.src_idx = rule->src_idx; r.gather = rule->gather;
-    r.out = out; r.viol = viol;
-    uint32_t want_in = 1;
-    switch (rule->kind) {
-    case GIFT_RULE_IDENTITY: break;
-    case GIFT_RULE_BROADCAST: if (!rule->gather && rule->n_out) return GIFT_E_INVAL; break;
-    case GIFT_RULE_ROWWISE:
-        if (rule->n_in < 1 || rule->n_in > 8) return GIFT_E_INVAL;
-        want_in = rule->n_in;
-        break;
-    case GIFT_RULE_SEGREDUCE:
-        if (rule->n_in != 2 || !rule->seg_ptr || !rule->src_ptr || (!rule->src_idx && rule->n_seg)) return GIFT_E_INVAL;
-        want_in = 2;
-        break;
-    default: return GIFT_E_INVAL;
-    }
-    if (rule->n_in != want_in) return GIFT_E_INVAL;
-    for (uint32_t k = 0; k < want_in; k++) {
-        if (!in_maps[k]) return GIFT_E_INVAL;
-        r.in[k] = in_maps[k];
-    }
+    const int rc = fill_rule_args(rule, in_maps, out, viol, r);
+    if (rc != GIFT_OK) return rc;
     DeviceGuard g(c->device);
     if (!g.ok) return GIFT_E_CUDA;
     cudaStream_t st = (cudaStream_t)stream;
