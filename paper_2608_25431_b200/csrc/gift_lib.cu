@@ -355,10 +355,18 @@ __global__ void __launch_bounds__(THREADS, 1) crypt_kernel(CallArgs a, const uin
         run = __shfl_sync(0xFFFFFFFFu, run, 0);
         if (run >= total_runs) break;
         // segment of this run: the largest s with run_prefix[s] <= run
+        // (the 32 lanes probe 32 points of the interval at once: 3-4 dependent loads, not 17)
         uint32_t lo = 0, hi = a.nseg;
         while (hi - lo > 1) {
-            const uint32_t mid = (lo + hi) >> 1;
-            if (a.run_prefix[mid] <= run) lo = mid; else hi = mid;
+            const uint32_t span = hi - lo - 1;                       // candidates lo+1 .. hi-1
+            const uint32_t step = span / 32u + 1u;
+            const uint32_t probe = lo + 1u + (uint32_t)lane * step;  // increasing with the lane
+            const bool le = probe < hi && a.run_prefix[probe] <= run;
+            const uint32_t m = __ballot_sync(0xFFFFFFFFu, le);       // true on a prefix of the lanes
+            const int k = __popc(m);
+            const uint32_t next = lo + 1u + (uint32_t)k * step;      // first probe that said "greater"
+            if (k) lo = lo + 1u + (uint32_t)(k - 1) * step;
+            if (k < 32 && next < hi) hi = next;
         }
         const uint32_t s = lo;
         const uint32_t first_run = a.run_prefix[s];
@@ -658,8 +666,10 @@ int seg_call(gift_ctx* c, const void* src, void* dst, uint64_t buf_bytes, const 
     a.ticket = c->d_ticket;
     a.glob = c->d_glob;
     a.resident_warps = (uint32_t)c->num_sms * (uint32_t)(c->threads / 32);
-    a.target_runs = a.resident_warps * 8u;                // about eight runs per resident warp
-    a.max_run_blocks = 4096u;                             // 64 KiB
+    // A run costs about two rows of 32 blocks beyond its own rows (pipeline fill, power
+    // fix-up, combining), so runs are long; about ten per resident warp keep the tail short.
+    a.target_runs = a.resident_warps * 10u;
+    a.max_run_blocks = 16384u;                            // 256 KiB
     a.min_run_blocks = 64u;                               // 1 KiB
 
     CU_TRY(cudaMemsetAsync(c->d_glob, 0, sizeof(Globals), st));
@@ -1038,8 +1048,8 @@ extern "C" int gift_seg_encrypt_static(gift_ctx* c, const void* src, void* dst, 
     a.acc = reinterpret_cast<uint4*>(scratch + STATIC_OFF_ACC);
     a.ticket = reinterpret_cast<uint32_t*>(scratch + STATIC_OFF_TICKET);
     a.resident_warps = (uint32_t)c->num_sms * (uint32_t)(c->threads / 32);
-    a.target_runs = a.resident_warps * 8u;
-    a.max_run_blocks = 4096u;
+    a.target_runs = a.resident_warps * 10u;
+    a.max_run_blocks = 16384u;
     a.min_run_blocks = 64u;
 
     // The array still holds the previous call's values: the counters are cleared here, the
