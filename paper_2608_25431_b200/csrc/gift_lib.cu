@@ -104,7 +104,7 @@ struct CallArgs {
     uint4* acc;
     uint32_t* ticket;
     Globals* glob;
-    uint32_t target_runs;          // runs wanted for a balanced call
+    uint32_t runs_per_warp;        // most runs a resident warp should get in a large call
     uint32_t resident_warps;       // warps of the cipher kernel on the whole GPU
     uint32_t max_run_blocks;
     uint32_t min_run_blocks;
@@ -217,13 +217,17 @@ __global__ void scan_kernel(CallArgs a)
     __shared__ uint32_t run_blocks_s;
     const int tid = threadIdx.x, lane = tid & 31, wid = tid >> 5;
     if (tid == 0) {
-        // Run length (a multiple of 32 blocks, so that rows stay aligned): large calls get about
-        // eight runs per resident warp, so that the dynamic hand-out evens out skewed segment
-        // lengths; calls too small for that get one run per warp, which avoids a second,
-        // mostly empty wave.
+        // Run length (a multiple of 32 blocks, so that rows stay aligned).  A run costs its warp
+        // about two rows beyond its own, so runs are long: a warp's share of the call is cut
+        // into one run per 4 096 blocks, at most runs_per_warp of them (enough for the dynamic
+        // hand-out to even out skewed segment lengths) and at least one (small calls: a second,
+        // mostly empty wave would cost more than any imbalance).
         const unsigned long long total = a.glob->total_blocks;
-        unsigned long long rb = (total + a.target_runs - 1) / a.target_runs;
-        if (rb < 512) rb = (total + a.resident_warps - 1) / a.resident_warps;
+        const unsigned long long per_warp = (total + a.resident_warps - 1) / a.resident_warps;
+        unsigned long long k = per_warp / 4096u;
+        if (k < 1) k = 1;
+        if (k > a.runs_per_warp) k = a.runs_per_warp;
+        unsigned long long rb = (per_warp + k - 1) / k;
         rb = (rb + 31) / 32 * 32;
         if (rb < a.min_run_blocks) rb = a.min_run_blocks;
         if (rb > a.max_run_blocks) rb = a.max_run_blocks;
@@ -373,9 +377,12 @@ __global__ void __launch_bounds__(THREADS, 1) crypt_kernel(CallArgs a, const uin
         const uint32_t seg_runs = a.run_prefix[s + 1] - first_run;
         const gift_seg seg = a.segs[s];
         const uint64_t nblk = seg_blocks(seg.len);
-        const uint64_t run_first = (uint64_t)(run - first_run) * run_blocks;
+        // the segment's runs are made equal: its block count divided by its run count, rounded
+        // up to whole rows (never more than run_blocks, and the last run is never empty)
+        const uint32_t seg_rb = seg_runs > 1 ? (uint32_t)(((nblk + seg_runs - 1) / seg_runs + 31) & ~(uint64_t)31) : run_blocks;
+        const uint64_t run_first = (uint64_t)(run - first_run) * seg_rb;
         const uint64_t left = nblk - run_first;
-        const uint32_t run_n = left < run_blocks ? (uint32_t)left : run_blocks;
+        const uint32_t run_n = left < seg_rb ? (uint32_t)left : seg_rb;
 
         // this warp's copy of the owner's key material (512 bytes: one uint4 per lane)
         __syncwarp();
@@ -666,9 +673,7 @@ int seg_call(gift_ctx* c, const void* src, void* dst, uint64_t buf_bytes, const 
     a.ticket = c->d_ticket;
     a.glob = c->d_glob;
     a.resident_warps = (uint32_t)c->num_sms * (uint32_t)(c->threads / 32);
-    // A run costs about two rows of 32 blocks beyond its own rows (pipeline fill, power
-    // fix-up, combining), so runs are long; about ten per resident warp keep the tail short.
-    a.target_runs = a.resident_warps * 10u;
+    a.runs_per_warp = 8u;
     a.max_run_blocks = 16384u;                            // 256 KiB
     a.min_run_blocks = 64u;                               // 1 KiB
 
@@ -1048,7 +1053,7 @@ extern "C" int gift_seg_encrypt_static(gift_ctx* c, const void* src, void* dst, 
     a.acc = reinterpret_cast<uint4*>(scratch + STATIC_OFF_ACC);
     a.ticket = reinterpret_cast<uint32_t*>(scratch + STATIC_OFF_TICKET);
     a.resident_warps = (uint32_t)c->num_sms * (uint32_t)(c->threads / 32);
-    a.target_runs = a.resident_warps * 10u;
+    a.runs_per_warp = 8u;
     a.max_run_blocks = 16384u;
     a.min_run_blocks = 64u;
 
