@@ -7,7 +7,7 @@ Workload (default): the prefill -> decode KV-cache handoff of a LLaMA-7B-shaped 
 (workloads.config3 at 32 layers): every 256 KiB KV block of every user encrypted under its
 owner's key with a per-block tag.  One step = one pass of the whole hot path over that
 batch: the four flow rules on the blocks' owner labels (copy, row-preserving, per-group
-reduction, scatter to pool pages; one fused launch), then gift_seg_encrypt (plan + label check, work list,
+reduction, scatter to pool pages; one fused launch), then gift_seg_encrypt (plan + label check, work split,
 CTR + GHASH, tag finish) in place.  Key
 setup is outside the step, as it is once per key change.  The path does not shard: with
 --gpus N every rank runs an independent replica on its own GPU (no collective on the data

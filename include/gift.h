@@ -156,7 +156,7 @@ int gift_seg_encrypt(gift_ctx* ctx, const void* src, void* dst, uint64_t buf_byt
  * scratch with cudaMalloc when a call has more segments than any before it; this entry
  * point never does.  It calls no cudaMalloc, cudaFree or other allocating routine: its
  * scratch (work list, partial hashes, counters) is a fixed array inside the library image,
- * about 1.6 MB, which every GPU that loads the library holds until the process exits.
+ * about 1.9 MB, which every GPU that loads the library holds until the process exits.
  *   - Arguments, results and status words are exactly those of gift_seg_encrypt; the ctx
  *     (created earlier, when allocation was still allowed) supplies the keys.
  *   - nseg must not exceed GIFT_STATIC_MAX_SEGS (65536); a larger table is refused with

@@ -220,7 +220,7 @@ GIFT_HD u128 run_lane_rows(const Tab& tb, const uint32_t* rk, const CtrPrefix& p
                            const u128* powtab, const uint8_t* src, uint8_t* dst, const SegAddr& addr,
                            uint64_t seg_nblk, uint64_t run_first, uint32_t run_n, uint32_t tail, int lane)
 {
-    const bool has_partial = tail != 0 && run_first + run_n == seg_nblk;
+    const bool has_partial = tail != 0 && run_n != 0 && run_first + run_n == seg_nblk;
     const uint32_t n_full = run_n - (has_partial ? 1u : 0u);
     const uint32_t rows = n_full >> 5;                      // rows in which all 32 lanes hold a full block
     u128 acc = gf_zero();

@@ -12,11 +12,9 @@
 // ---------------------------------------------------------------------------
 
 struct Globals {
-    unsigned long long total_blocks;   // 16-byte blocks of all accepted segments
-    uint32_t total_runs;
-    uint32_t run_blocks;               // blocks per run chosen for this call
-    uint32_t work;                     // next run to hand out
-    uint32_t pad[3];
+    unsigned long long total_weight;   // sum of the accepted segments' weights (see scan_kernel)
+    unsigned long long slice;          // weight handed to each resident warp
+    uint32_t pad[4];
 };
 
 struct gift_ctx {
@@ -36,7 +34,7 @@ struct gift_ctx {
     int32_t* d_stage_ids;
     uint8_t* d_stage_keys;
     uint32_t seg_cap;
-    uint32_t* d_run_prefix;            // [seg_cap + 1]
+    unsigned long long* d_wprefix;     // [seg_cap + 1] exclusive prefix of the segment weights
     uint4* d_acc;                      // [seg_cap]
     uint32_t* d_ticket;                // [seg_cap]
     Globals* d_glob;

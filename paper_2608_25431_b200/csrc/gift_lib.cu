@@ -3,12 +3,12 @@
 // Call structure of gift_seg_encrypt / gift_seg_decrypt / gift_verify_tags, all
 // on the caller's stream with no host round trip in between:
 //   1. plan_kernel     one warp per segment: descriptor checks, ownership-label
-//                      check, pre-status, zeroed hash accumulators, block total
-//   2. scan_kernel     picks the run length from the block total and turns runs
-//                      per segment into a prefix sum (the work list)
-//   3. crypt_kernel    persistent warps pull runs from a counter; per run:
-//                      CTR keystream + XOR + GHASH; the warp that completes a
-//                      segment finishes its tag (no waiting, tickets only)
+//                      check, pre-status, zeroed hash accumulators
+//   2. scan_kernel     prefix sum of the accepted segments' weights and the weight
+//                      slice of a resident warp (the static work split)
+//   3. crypt_kernel    every resident warp takes its slice; per piece of a segment:
+//                      CTR keystream + XOR + GHASH; the warp whose report completes
+//                      a segment finishes its tag (no waiting, tickets only)
 //   4. fixup_kernel    decrypt only: zero-fills failed segments, marks their units
 //
 // AES uses T-tables replicated across the 32 shared-memory banks so that a warp's
@@ -100,14 +100,11 @@ struct CallArgs {
     const KeyHot* hot;
     const u128* pow;
     uint32_t max_users;
-    uint32_t* run_prefix;
+    unsigned long long* wprefix;   // [nseg + 1] exclusive prefix of the segment weights
     uint4* acc;
     uint32_t* ticket;
     Globals* glob;
-    uint32_t runs_per_warp;        // most runs a resident warp should get in a large call
     uint32_t resident_warps;       // warps of the cipher kernel on the whole GPU
-    uint32_t max_run_blocks;
-    uint32_t min_run_blocks;
 };
 
 __device__ __forceinline__ uint64_t seg_blocks(uint64_t len) { return (len + 15) >> 4; }
@@ -189,84 +186,81 @@ __global__ void plan_kernel(CallArgs a)
         a.status[s] = st;
         a.acc[s] = make_uint4(0u, 0u, 0u, 0u);
         a.ticket[s] = 0u;
-        if (st == 0) {
-            const uint64_t nb = seg_blocks(seg.len);
-            atomicAdd(&a.glob->total_blocks, (unsigned long long)(nb ? nb : 1));
-        } else if (MODE == MODE_ENCRYPT) {
+        if (st != 0 && MODE == MODE_ENCRYPT) {
             reinterpret_cast<uint4*>(a.tags)[s] = make_uint4(0u, 0u, 0u, 0u);
         }
     }
 }
 
 // ---------------------------------------------------------------------------
-// 2. scan: run length and work list
+// 2. scan: the work split
 // ---------------------------------------------------------------------------
+//
+// The cost of a block does not depend on the data, so the call is split statically: every
+// accepted segment gets a weight, the weights are laid end to end, and resident warp w takes
+// the weight range [w*slice, (w+1)*slice).  A segment's weight is its rows of 32 blocks plus
+// SEG_WEIGHT for what a piece of work costs beyond its rows (pipeline fill, power fix-up, tag:
+// about two rows, measured); its first SEG_WEIGHT units stand for that overhead, the rest
+// map to its blocks.  A slice boundary inside a segment is rounded down to a whole row, so
+// every warp's piece of a segment starts on a row.  Nothing is handed out at run time: no
+// work counter, no imbalance from partial waves, and a warp touches as few segments as can be.
 
-__device__ __forceinline__ uint32_t runs_of(uint64_t len, uint32_t st, uint32_t run_blocks)
+constexpr uint32_t SEG_WEIGHT = 64u;
+constexpr uint32_t MIN_SLICE = 256u;      // small calls: fewer warps rather than thinner slices
+
+__device__ __forceinline__ unsigned long long weight_of(uint64_t len, uint32_t st)
 {
-    if (st != 0) return 0u;
-    const uint64_t nb = seg_blocks(len);
-    const uint64_t r = (nb + run_blocks - 1) / run_blocks;
-    return r ? (uint32_t)r : 1u;      // an empty segment still needs its tag finished
+    if (st != 0) return 0ull;
+    return ((seg_blocks(len) + 31u) & ~(uint64_t)31u) + SEG_WEIGHT;   // an empty segment still needs its tag
+}
+
+// First block of the piece that starts at weight distance d from the segment's start.
+__device__ __forceinline__ uint64_t slice_cut(uint64_t d, uint64_t nblk)
+{
+    if (d <= SEG_WEIGHT) return 0;
+    const uint64_t b = d - SEG_WEIGHT;
+    return b >= nblk ? nblk : (b & ~(uint64_t)31u);
 }
 
 __global__ void scan_kernel(CallArgs a)
 {
-    __shared__ uint32_t warp_sums[32];
-    __shared__ uint32_t carry;
-    __shared__ uint32_t run_blocks_s;
+    __shared__ unsigned long long warp_sums[32];
+    __shared__ unsigned long long carry;
     const int tid = threadIdx.x, lane = tid & 31, wid = tid >> 5;
-    if (tid == 0) {
-        // Run length (a multiple of 32 blocks, so that rows stay aligned).  A run costs its warp
-        // about two rows beyond its own, so runs are long: a warp's share of the call is cut
-        // into one run per 4 096 blocks, at most runs_per_warp of them (enough for the dynamic
-        // hand-out to even out skewed segment lengths) and at least one (small calls: a second,
-        // mostly empty wave would cost more than any imbalance).
-        const unsigned long long total = a.glob->total_blocks;
-        const unsigned long long per_warp = (total + a.resident_warps - 1) / a.resident_warps;
-        unsigned long long k = per_warp / 4096u;
-        if (k < 1) k = 1;
-        if (k > a.runs_per_warp) k = a.runs_per_warp;
-        unsigned long long rb = (per_warp + k - 1) / k;
-        rb = (rb + 31) / 32 * 32;
-        if (rb < a.min_run_blocks) rb = a.min_run_blocks;
-        if (rb > a.max_run_blocks) rb = a.max_run_blocks;
-        run_blocks_s = (uint32_t)rb;
-        carry = 0u;
-    }
+    if (tid == 0) carry = 0ull;
     __syncthreads();
-    const uint32_t rb = run_blocks_s;
     for (uint32_t base = 0; base < a.nseg; base += blockDim.x) {
         const uint32_t i = base + tid;
-        uint32_t v = 0;
-        if (i < a.nseg) v = runs_of(a.segs[i].len, a.status[i], rb);
-        uint32_t x = v;
+        unsigned long long v = 0;
+        if (i < a.nseg) v = weight_of(a.segs[i].len, a.status[i]);
+        unsigned long long x = v;
         for (int o = 1; o < 32; o <<= 1) {
-            const uint32_t y = __shfl_up_sync(0xFFFFFFFFu, x, o);
+            const unsigned long long y = __shfl_up_sync(0xFFFFFFFFu, x, o);
             if (lane >= o) x += y;
         }
         if (lane == 31) warp_sums[wid] = x;
         __syncthreads();
         if (wid == 0) {
-            uint32_t w = lane < (int)(blockDim.x >> 5) ? warp_sums[lane] : 0u;
+            unsigned long long w = lane < (int)(blockDim.x >> 5) ? warp_sums[lane] : 0ull;
             for (int o = 1; o < 32; o <<= 1) {
-                const uint32_t y = __shfl_up_sync(0xFFFFFFFFu, w, o);
+                const unsigned long long y = __shfl_up_sync(0xFFFFFFFFu, w, o);
                 if (lane >= o) w += y;
             }
             warp_sums[lane] = w;      // inclusive sums of the warps
         }
         __syncthreads();
-        const uint32_t before = carry + (wid ? warp_sums[wid - 1] : 0u) + (x - v);
-        if (i < a.nseg) a.run_prefix[i] = before;
+        const unsigned long long before = carry + (wid ? warp_sums[wid - 1] : 0ull) + (x - v);
+        if (i < a.nseg) a.wprefix[i] = before;
         __syncthreads();
         if (tid == 0) carry += warp_sums[(blockDim.x >> 5) - 1];
         __syncthreads();
     }
     if (tid == 0) {
-        a.run_prefix[a.nseg] = carry;
-        a.glob->total_runs = carry;
-        a.glob->run_blocks = rb;
-        a.glob->work = 0u;
+        a.wprefix[a.nseg] = carry;
+        unsigned long long slice = (carry + a.resident_warps - 1) / a.resident_warps;
+        if (slice < MIN_SLICE) slice = MIN_SLICE;
+        a.glob->total_weight = carry;
+        a.glob->slice = slice;
     }
 }
 
@@ -351,38 +345,42 @@ __global__ void __launch_bounds__(THREADS, 1) crypt_kernel(CallArgs a, const uin
     tb.lb1 = (uint32_t)lane * 4u + 128u;
     KeyHot* slot = reinterpret_cast<KeyHot*>(smem_raw + TAB_BYTES) + wid;
 
-    const uint32_t total_runs = a.glob->total_runs;
-    const uint32_t run_blocks = a.glob->run_blocks;
-    for (;;) {
-        uint32_t run = 0;
-        if (lane == 0) run = atomicAdd(&a.glob->work, 1u);
-        run = __shfl_sync(0xFFFFFFFFu, run, 0);
-        if (run >= total_runs) break;
-        // segment of this run: the largest s with run_prefix[s] <= run
-        // (the 32 lanes probe 32 points of the interval at once: 3-4 dependent loads, not 17)
+    // this warp's share of the call: the weight range [g0, g1) (see scan_kernel)
+    const uint64_t total_weight = a.glob->total_weight, slice = a.glob->slice;
+    const uint64_t g0 = (uint64_t)(blockIdx.x * (THREADS / 32) + wid) * slice;
+    if (g0 >= total_weight) return;
+    const uint64_t g1 = g0 + slice < total_weight ? g0 + slice : total_weight;
+    // first segment: the largest s with wprefix[s] <= g0 (among equal prefixes the last one, which
+    // is the one that has weight); the 32 lanes probe 32 points of the interval per step
+    uint32_t s;
+    {
         uint32_t lo = 0, hi = a.nseg;
         while (hi - lo > 1) {
             const uint32_t span = hi - lo - 1;                       // candidates lo+1 .. hi-1
             const uint32_t step = span / 32u + 1u;
             const uint32_t probe = lo + 1u + (uint32_t)lane * step;  // increasing with the lane
-            const bool le = probe < hi && a.run_prefix[probe] <= run;
+            const bool le = probe < hi && a.wprefix[probe] <= g0;
             const uint32_t m = __ballot_sync(0xFFFFFFFFu, le);       // true on a prefix of the lanes
             const int k = __popc(m);
             const uint32_t next = lo + 1u + (uint32_t)k * step;      // first probe that said "greater"
             if (k) lo = lo + 1u + (uint32_t)(k - 1) * step;
             if (k < 32 && next < hi) hi = next;
         }
-        const uint32_t s = lo;
-        const uint32_t first_run = a.run_prefix[s];
-        const uint32_t seg_runs = a.run_prefix[s + 1] - first_run;
+        s = lo;
+    }
+    for (; s < a.nseg; s++) {
+        const uint64_t p0 = a.wprefix[s];
+        if (p0 >= g1) break;
+        const uint64_t p1 = a.wprefix[s + 1];
+        if (p1 == p0) continue;                                      // rejected by the plan: no weight
         const gift_seg seg = a.segs[s];
         const uint64_t nblk = seg_blocks(seg.len);
-        // the segment's runs are made equal: its block count divided by its run count, rounded
-        // up to whole rows (never more than run_blocks, and the last run is never empty)
-        const uint32_t seg_rb = seg_runs > 1 ? (uint32_t)(((nblk + seg_runs - 1) / seg_runs + 31) & ~(uint64_t)31) : run_blocks;
-        const uint64_t run_first = (uint64_t)(run - first_run) * seg_rb;
-        const uint64_t left = nblk - run_first;
-        const uint32_t run_n = left < seg_rb ? (uint32_t)left : seg_rb;
+        // this warp's piece of the segment, and how many warps have one (each reports once,
+        // with or without blocks; the last report finishes the tag)
+        const uint64_t run_first = g0 <= p0 ? 0 : slice_cut(g0 - p0, nblk);
+        const uint64_t run_end = g1 >= p1 ? nblk : slice_cut(g1 - p0, nblk);
+        const uint32_t run_n = (uint32_t)(run_end - run_first);
+        const uint32_t seg_runs = (g0 <= p0 && g1 >= p1) ? 1u : (uint32_t)((p1 - 1) / slice - p0 / slice) + 1u;
 
         // this warp's copy of the owner's key material (512 bytes: one uint4 per lane)
         __syncwarp();
@@ -399,8 +397,11 @@ __global__ void __launch_bounds__(THREADS, 1) crypt_kernel(CallArgs a, const uin
         addr.page_bytes = a.page_bytes;
         addr.origin = a.page_table ? (uint64_t)seg.page0 : seg.offset;
 
-        u128 part;
-        if (U == 1 && (a.page_table == nullptr || (a.page_bytes & 511) == 0)) {
+        u128 part = gf_zero();
+        if (run_n == 0) {
+            // a piece without blocks (an empty segment, or a slice boundary inside the segment's
+            // overhead weight or its last partial row): nothing to read, only the report below
+        } else if (U == 1 && (a.page_table == nullptr || (a.page_bytes & 511) == 0)) {
             // rows of 32 blocks never straddle a page: the pipelined row loop applies
             part = run_lane_rows<MODE>(tb, rk, pre, slot->hs[0], a.pow + (size_t)seg.owner * (POW_LEVELS * 256),
                                        a.src, a.dst, addr, nblk, run_first, run_n, (uint32_t)(seg.len & 15), lane);
@@ -584,12 +585,12 @@ int ensure_scratch(gift_ctx* c, uint32_t nseg)
     uint32_t cap = c->seg_cap ? c->seg_cap : 1024u;
     while (cap < nseg) cap = cap > 0x7FFFFFFFu ? nseg : cap * 2u;
     CU_TRY(cudaDeviceSynchronize());
-    cudaFree(c->d_run_prefix);
+    cudaFree(c->d_wprefix);
     cudaFree(c->d_acc);
     cudaFree(c->d_ticket);
-    c->d_run_prefix = nullptr; c->d_acc = nullptr; c->d_ticket = nullptr;
+    c->d_wprefix = nullptr; c->d_acc = nullptr; c->d_ticket = nullptr;
     c->seg_cap = 0;
-    CU_TRY(cudaMalloc(&c->d_run_prefix, ((size_t)cap + 1) * sizeof(uint32_t)));
+    CU_TRY(cudaMalloc(&c->d_wprefix, ((size_t)cap + 1) * sizeof(unsigned long long)));
     CU_TRY(cudaMalloc(&c->d_acc, (size_t)cap * sizeof(uint4)));
     CU_TRY(cudaMalloc(&c->d_ticket, (size_t)cap * sizeof(uint32_t)));
     c->seg_cap = cap;
@@ -668,14 +669,11 @@ int seg_call(gift_ctx* c, const void* src, void* dst, uint64_t buf_bytes, const 
     a.hot = c->d_hot;
     a.pow = c->d_pow;
     a.max_users = c->max_users;
-    a.run_prefix = c->d_run_prefix;
+    a.wprefix = c->d_wprefix;
     a.acc = c->d_acc;
     a.ticket = c->d_ticket;
     a.glob = c->d_glob;
     a.resident_warps = (uint32_t)c->num_sms * (uint32_t)(c->threads / 32);
-    a.runs_per_warp = 8u;
-    a.max_run_blocks = 16384u;                            // 256 KiB
-    a.min_run_blocks = 64u;                               // 1 KiB
 
     CU_TRY(cudaMemsetAsync(c->d_glob, 0, sizeof(Globals), st));
     const uint32_t plan_blocks = (nseg + 7) / 8;          // 8 warps per block, one warp per segment
@@ -757,7 +755,7 @@ int gift_ctx_destroy(gift_ctx* c)
         if (c->d_stage_keys) cudaMemset(c->d_stage_keys, 0, (size_t)c->stage_cap * 16);
         cudaDeviceSynchronize();
         cudaFree(c->d_t0); cudaFree(c->d_isbox); cudaFree(c->d_hot); cudaFree(c->d_pow); cudaFree(c->d_glob);
-        cudaFree(c->d_run_prefix); cudaFree(c->d_acc); cudaFree(c->d_ticket);
+        cudaFree(c->d_wprefix); cudaFree(c->d_acc); cudaFree(c->d_ticket);
         cudaFree(c->d_stage_ids); cudaFree(c->d_stage_keys); cudaFree(c->d_snapshot); cudaFree(c->d_next_sync);
         if (c->h_stage) {
             memset(c->h_stage, 0, (size_t)c->stage_cap * 20);
@@ -986,7 +984,7 @@ uint64_t gift_launch_count(const gift_ctx* c) { return c ? c->launches : 0; }
 namespace {
 
 constexpr size_t STATIC_OFF_PREFIX = 256;                                                   // after Globals
-constexpr size_t STATIC_OFF_ACC = STATIC_OFF_PREFIX + ((size_t)GIFT_STATIC_MAX_SEGS + 64) * 4;   // 16-byte aligned
+constexpr size_t STATIC_OFF_ACC = STATIC_OFF_PREFIX + ((size_t)GIFT_STATIC_MAX_SEGS + 64) * 8;   // 16-byte aligned
 constexpr size_t STATIC_OFF_TICKET = STATIC_OFF_ACC + (size_t)GIFT_STATIC_MAX_SEGS * 16;
 constexpr size_t STATIC_SCRATCH_BYTES = STATIC_OFF_TICKET + (size_t)GIFT_STATIC_MAX_SEGS * 4;
 static_assert(sizeof(Globals) <= STATIC_OFF_PREFIX && STATIC_OFF_ACC % 16 == 0, "static scratch layout");
@@ -1049,16 +1047,13 @@ extern "C" int gift_seg_encrypt_static(gift_ctx* c, const void* src, void* dst, 
     a.pow = c->d_pow;
     a.max_users = c->max_users;
     a.glob = reinterpret_cast<Globals*>(scratch);
-    a.run_prefix = reinterpret_cast<uint32_t*>(scratch + STATIC_OFF_PREFIX);
+    a.wprefix = reinterpret_cast<unsigned long long*>(scratch + STATIC_OFF_PREFIX);
     a.acc = reinterpret_cast<uint4*>(scratch + STATIC_OFF_ACC);
     a.ticket = reinterpret_cast<uint32_t*>(scratch + STATIC_OFF_TICKET);
     a.resident_warps = (uint32_t)c->num_sms * (uint32_t)(c->threads / 32);
-    a.runs_per_warp = 8u;
-    a.max_run_blocks = 16384u;
-    a.min_run_blocks = 64u;
 
     // The array still holds the previous call's values: the counters are cleared here, the
-    // per-segment accumulators and tickets by the plan kernel, the work list by the scan kernel.
+    // per-segment accumulators and tickets by the plan kernel, the weight prefix by the scan kernel.
     CU_TRY(cudaMemsetAsync(a.glob, 0, sizeof(Globals), st));
     plan_kernel<MODE_ENCRYPT><<<(nseg + 7) / 8, 256, 0, st>>>(a);
     scan_kernel<<<1, 1024, 0, st>>>(a);
