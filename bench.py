@@ -42,7 +42,7 @@ UNIT = "GB/s"
 # DRAM bytes per payload byte of the cipher kernel, from the ncu capture summarised in
 # profiles/crypt_kernel_c3_2layers.md (dram__bytes_read.sum + dram__bytes_write.sum over the
 # payload of that launch); traffic grows in proportion to the payload.
-NCU_DRAM_BYTES_PER_PAYLOAD_BYTE = 1.931
+NCU_DRAM_BYTES_PER_PAYLOAD_BYTE = 1.919
 
 FIRST_ALU_OPS_PER_BLOCK = 660
 ALU_OPS_PER_BLOCK = 483          # logic / permute / shift lane-operations (the binding pipe)
