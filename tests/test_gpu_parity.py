@@ -122,6 +122,30 @@ def test_large_segments_many_runs_and_high_powers():
     _roundtrip_exact(w, in_place=True)
 
 
+def test_one_segment_beyond_2_pow_24_blocks_uses_the_top_power_level():
+    """256 MiB + 4 KiB + 5 bytes in one segment: the first blocks' exponents exceed 2^24, the
+    fourth digit of the power table, which no workload of the paper's sizes reaches."""
+    rng = np.random.default_rng(13)
+    n = (256 << 20) + 4096 + 5
+    segs = np.zeros(1, dtype=W.SEG_DTYPE)
+    segs["owner"], segs["offset"], segs["len"] = 1, 0, n
+    segs["nonce"] = np.frombuffer(rng.bytes(12), dtype=np.uint8).reshape(1, 12)
+    ids, keys = np.arange(2, dtype=np.int32), np.frombuffer(rng.bytes(32), dtype=np.uint8).reshape(2, 16)
+    buf = np.frombuffer(rng.bytes((n + 15) // 16 * 16), dtype=np.uint8).copy()
+    w = W.Workload("huge", ids, keys, 2, buf, buf.size, segs)
+    ctx = make_ctx(w)
+    d = dev(w.buf)
+    tags, st = gpu_encrypt(ctx, w, d)
+    ref_ct = w.buf.copy()
+    ref_tags, ref_st = oracle_encrypt(w, w.buf, ref_ct)            # one oracle pass: about 20 s on one core
+    assert not ref_st.any() and not st_(st).any()
+    assert np.array_equal(np_(tags), ref_tags)
+    assert np.array_equal(np_(d), ref_ct)
+    st2 = gpu_decrypt(ctx, w, d, tags)                             # and back, against the original bytes
+    assert not st_(st2).any() and np.array_equal(np_(d), w.buf)
+    ctx.close()
+
+
 def test_export_status_rules_match_oracle():
     w = W.config2(n_users=8, vocab=64)
     om = w.owner_map.copy()
