@@ -356,8 +356,63 @@ __device__ __forceinline__ uint32_t warp_xor(uint32_t v)
     return v;
 }
 
+// Segments whose hash is complete wait here, per warp, until 32 of them can be finished at
+// once.  Finishing a tag is one cipher block (E_K(J0)) and one field multiply (LEN * H) per
+// segment; done right away it would occupy a whole warp for one segment's worth of work.  With
+// one segment per lane the same instructions finish 32 tags, each lane reading its own
+// segment's key material from global memory (the table lookups stay conflict-free: a lane
+// always reads its own bank's copy).
+struct Pending {
+    uint4 sum[32];
+    uint32_t seg[32];
+};
+
+template <int MODE, class Tab>
+__device__ __noinline__ void finish_pending(const CallArgs& a, const Tab& tb, const Pending* pend, uint32_t n, int lane)
+{
+    bool ok = false;
+    uint32_t s = 0;
+    if ((uint32_t)lane < n) {
+        s = pend->seg[lane];
+        const uint4 sv = pend->sum[lane];
+        const gift_seg seg = a.segs[s];
+        const KeyHot* hk = a.hot + seg.owner;
+        u128 sum;
+        sum.w[0] = sv.x; sum.w[1] = sv.y; sum.w[2] = sv.z; sum.w[3] = sv.w;
+        uint32_t nonce[3];
+        nonce[0] = (uint32_t)seg.nonce[0] | ((uint32_t)seg.nonce[1] << 8) | ((uint32_t)seg.nonce[2] << 16) | ((uint32_t)seg.nonce[3] << 24);
+        nonce[1] = (uint32_t)seg.nonce[4] | ((uint32_t)seg.nonce[5] << 8) | ((uint32_t)seg.nonce[6] << 16) | ((uint32_t)seg.nonce[7] << 24);
+        nonce[2] = (uint32_t)seg.nonce[8] | ((uint32_t)seg.nonce[9] << 8) | ((uint32_t)seg.nonce[10] << 16) | ((uint32_t)seg.nonce[11] << 24);
+        uint32_t tag[4];
+        finish_tag(tb, hk->rk, hk->h, nonce, seg.len, sum, tag, a.aad ? a.aad + 16 * (size_t)s : nullptr,
+                   a.pow + (size_t)seg.owner * (POW_LEVELS * 256));
+        uint4* tagp = reinterpret_cast<uint4*>(a.tags) + s;
+        if (MODE == MODE_ENCRYPT) {
+            *tagp = make_uint4(tag[0], tag[1], tag[2], tag[3]);
+        } else {
+            const uint4 given = *tagp;
+            ok = given.x == tag[0] && given.y == tag[1] && given.z == tag[2] && given.w == tag[3];
+            if (!ok) a.status[s] = GIFT_ST_TAG_MISMATCH;
+        }
+    }
+    if (MODE == MODE_DECRYPT && a.owner_map != nullptr) {
+        // import succeeded: record the claimed owner on the covered units, the warp taking
+        // one verified segment at a time
+        uint32_t m = __ballot_sync(0xFFFFFFFFu, ok);
+        while (m) {
+            const int k = __ffs(m) - 1;
+            m &= m - 1;
+            const uint32_t sk = __shfl_sync(0xFFFFFFFFu, s, k);
+            const gift_seg seg = a.segs[sk];
+            uint64_t u0;
+            const uint64_t nu = seg_unit_count(a, seg, &u0);
+            for (uint64_t u = lane; u < nu; u += 32) a.owner_map[seg_unit(a, seg, u0, u)] = seg.owner;
+        }
+    }
+}
+
 template <int U, int MODE, int NT, int THREADS>
-__global__ void __launch_bounds__(THREADS, 1) crypt_kernel(CallArgs a, const uint32_t* __restrict__ t0)
+__global__ void __launch_bounds__(THREADS, 1) crypt_kernel(const __grid_constant__ CallArgs a, const uint32_t* __restrict__ t0)
 {
     constexpr uint32_t TAB_BYTES = NT == 4 ? 131072u : 65536u;
     const int lane = threadIdx.x & 31, wid = threadIdx.x >> 5;
@@ -367,6 +422,8 @@ __global__ void __launch_bounds__(THREADS, 1) crypt_kernel(CallArgs a, const uin
     tb.lb0 = (uint32_t)lane * 4u;
     tb.lb1 = (uint32_t)lane * 4u + 128u;
     KeyHot* slot = reinterpret_cast<KeyHot*>(smem_raw + TAB_BYTES) + wid;
+    Pending* pend = reinterpret_cast<Pending*>(smem_raw + TAB_BYTES + (THREADS / 32) * sizeof(KeyHot)) + wid;
+    uint32_t n_pend = 0;
 
     // this warp's share of the call: the weight range [g0, g1) (see scan_kernel)
     const uint64_t total_weight = a.glob->total_weight, slice = a.glob->slice;
@@ -465,25 +522,21 @@ __global__ void __launch_bounds__(THREADS, 1) crypt_kernel(CallArgs a, const uin
             }
         }
         if (last) {
-            uint32_t tag[4];
-            finish_tag(tb, rk, slot->h, nonce, seg.len, sum, tag, a.aad ? a.aad + 16 * (size_t)s : nullptr,
-                       a.pow + (size_t)seg.owner * (POW_LEVELS * 256));
-            uint4* tagp = reinterpret_cast<uint4*>(a.tags) + s;
-            if (MODE == MODE_ENCRYPT) {
-                if (lane == 0) *tagp = make_uint4(tag[0], tag[1], tag[2], tag[3]);
-            } else {
-                const uint4 given = *tagp;
-                const bool ok = given.x == tag[0] && given.y == tag[1] && given.z == tag[2] && given.w == tag[3];
-                if (lane == 0 && !ok) a.status[s] = GIFT_ST_TAG_MISMATCH;
-                if (MODE == MODE_DECRYPT && ok && a.owner_map != nullptr) {
-                    // import succeeded: record the claimed owner on the covered units
-                    uint64_t u0;
-                    const uint64_t nu = seg_unit_count(a, seg, &u0);
-                    for (uint64_t k = lane; k < nu; k += 32) a.owner_map[seg_unit(a, seg, u0, k)] = seg.owner;
-                }
+            if (lane == 0) {
+                pend->sum[n_pend] = make_uint4(sum.w[0], sum.w[1], sum.w[2], sum.w[3]);
+                pend->seg[n_pend] = s;
+            }
+            n_pend++;
+            if (n_pend == 32u) {
+                __syncwarp();
+                finish_pending<MODE>(a, tb, pend, n_pend, lane);
+                __syncwarp();
+                n_pend = 0;
             }
         }
     }
+    __syncwarp();
+    if (n_pend) finish_pending<MODE>(a, tb, pend, n_pend, lane);
 }
 
 // ---------------------------------------------------------------------------
@@ -623,7 +676,7 @@ int ensure_scratch(gift_ctx* c, uint32_t nseg)
 template <int U, int MODE, int NT, int THREADS>
 int launch_crypt_t(gift_ctx* c, const CallArgs& a, cudaStream_t st)
 {
-    const size_t smem = (NT == 4 ? 131072u : 65536u) + (THREADS / 32) * sizeof(KeyHot);
+    const size_t smem = (NT == 4 ? 131072u : 65536u) + (THREADS / 32) * (sizeof(KeyHot) + sizeof(Pending));
     static bool configured[8] = {false, false, false, false, false, false, false, false};
     auto kern = crypt_kernel<U, MODE, NT, THREADS>;
     if (c->device < 8 && !configured[c->device]) {
