@@ -264,6 +264,8 @@ GIFT_HD u128 run_lane_rows(const Tab& tb, const uint32_t* rk, const CtrPrefix& p
         acc = xor128(gfmul(acc, hs), block_to_field(c_prev.d[0], c_prev.d[1], c_prev.d[2], c_prev.d[3]));
         c_prev = c;
         pending = true;
+        // (the advance stays behind the hash update: its branch would otherwise split the block in
+        // which the compiler interleaves cipher and hash; measured 405 instead of 436 GB/s)
         ctr += 32;
         off += 512;
         if (--rows_in_page == 0) {                          // next page (uniform across the warp)
