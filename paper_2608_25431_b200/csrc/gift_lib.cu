@@ -383,8 +383,16 @@ __device__ __noinline__ void finish_pending(const CallArgs& a, const Tab& tb, co
         nonce[0] = (uint32_t)seg.nonce[0] | ((uint32_t)seg.nonce[1] << 8) | ((uint32_t)seg.nonce[2] << 16) | ((uint32_t)seg.nonce[3] << 24);
         nonce[1] = (uint32_t)seg.nonce[4] | ((uint32_t)seg.nonce[5] << 8) | ((uint32_t)seg.nonce[6] << 16) | ((uint32_t)seg.nonce[7] << 24);
         nonce[2] = (uint32_t)seg.nonce[8] | ((uint32_t)seg.nonce[9] << 8) | ((uint32_t)seg.nonce[10] << 16) | ((uint32_t)seg.nonce[11] << 24);
+        // the lane's round keys and hash subkey in one batch of loads (read one by one as the
+        // rounds need them, their latency would sit on the tail of every call)
+        uint32_t rkl[48];
+#pragma unroll
+        for (int q = 0; q < 12; q++) {
+            const uint4 v = reinterpret_cast<const uint4*>(hk)[q];      // rk[0..43], then h[0..3]
+            rkl[4 * q] = v.x; rkl[4 * q + 1] = v.y; rkl[4 * q + 2] = v.z; rkl[4 * q + 3] = v.w;
+        }
         uint32_t tag[4];
-        finish_tag(tb, hk->rk, hk->h, nonce, seg.len, sum, tag, a.aad ? a.aad + 16 * (size_t)s : nullptr,
+        finish_tag(tb, rkl, rkl + 44, nonce, seg.len, sum, tag, a.aad ? a.aad + 16 * (size_t)s : nullptr,
                    a.pow + (size_t)seg.owner * (POW_LEVELS * 256));
         uint4* tagp = reinterpret_cast<uint4*>(a.tags) + s;
         if (MODE == MODE_ENCRYPT) {
