@@ -111,3 +111,35 @@ def test_many_tiny_segments():
     st2 = gpu_decrypt(ctx, w, d, tags)
     assert not st_(st2).any() and np.array_equal(np_(d), buf)
     ctx.close()
+
+
+def test_mid_size_flat_table_with_ragged_lengths():
+    """3 000 flat segments of 0..300 000 bytes (any byte length): about 450 MB, so that every
+    resident warp gets a slice of a few thousand blocks whose ends fall at arbitrary places
+    inside segments with partial last rows and partial last blocks."""
+    rng = np.random.default_rng(4242)
+    nseg, n_users = 3000, 7
+    lens = rng.integers(0, 300_001, size=nseg)
+    lens[rng.choice(nseg, size=40, replace=False)] = 0
+    offs = np.concatenate([[0], np.cumsum((lens + 15) // 16 * 16)[:-1]])
+    segs = np.zeros(nseg, dtype=W.SEG_DTYPE)
+    segs["owner"] = rng.integers(0, n_users, size=nseg)
+    segs["offset"] = offs
+    segs["len"] = lens
+    segs["nonce"] = np.frombuffer(rng.bytes(12 * nseg), dtype=np.uint8).reshape(nseg, 12)
+    ids = np.arange(n_users, dtype=np.int32)
+    keys = np.frombuffer(rng.bytes(16 * n_users), dtype=np.uint8).reshape(n_users, 16).copy()
+    total = int(offs[-1] + (lens[-1] + 15) // 16 * 16) + 64
+    buf = rng.integers(0, 256, size=total, dtype=np.uint8)
+    w = W.Workload("mid_flat", ids, keys, n_users, buf, buf.size, segs)
+    ctx = make_ctx(w)
+    d = dev(w.buf)
+    tags, st = gpu_encrypt(ctx, w, d)
+    ref = w.buf.copy()
+    ref_tags, ref_st = gcm.seg_encrypt(ref, ref, w.segs, ids, keys, n_users)
+    assert not ref_st.any() and not st_(st).any()
+    assert np.array_equal(np_(tags), ref_tags)
+    assert np.array_equal(np_(d), ref)
+    st2 = gpu_decrypt(ctx, w, d, tags)
+    assert not st_(st2).any() and np.array_equal(np_(d), w.buf)
+    ctx.close()
