@@ -48,6 +48,46 @@ GIFT_HD u128 mul_by_power(const u128& a, const u128* powtab, uint64_t e)
     return r;
 }
 
+// ---- static work split --------------------------------------------------------------------
+//
+// The accepted segments' weights are laid end to end and resident warp w takes the weight
+// range [w*slice, (w+1)*slice).  A segment's weight is its rows of 32 blocks plus SEG_WEIGHT
+// for what a piece of work costs beyond its rows; its first SEG_WEIGHT units stand for that
+// overhead, the rest map to its blocks.  A slice boundary inside a segment is rounded down to
+// a whole row, so every piece starts on a row.
+constexpr uint32_t SEG_WEIGHT = 64u;
+constexpr uint32_t MIN_SLICE = 256u;
+
+GIFT_HD uint64_t seg_weight(uint64_t nblk)
+{
+    return ((nblk + 31u) & ~(uint64_t)31u) + SEG_WEIGHT;     // an empty segment still needs its tag
+}
+
+// First block of the piece that starts at weight distance d from the segment's start.
+GIFT_HD uint64_t slice_cut(uint64_t d, uint64_t nblk)
+{
+    if (d <= SEG_WEIGHT) return 0;
+    const uint64_t b = d - SEG_WEIGHT;
+    return b >= nblk ? nblk : (b & ~(uint64_t)31u);
+}
+
+// The blocks [first, end) of a segment that belong to the slice [g0, g1), for a segment of nblk
+// blocks whose weight range is [p0, p1), and the number of slices that meet the segment: each
+// of those reports once, with or without blocks, and the last report completes the segment.
+struct SlicePiece {
+    uint64_t first, end;
+    uint32_t reporters;
+};
+
+GIFT_HD SlicePiece slice_piece(uint64_t g0, uint64_t g1, uint64_t p0, uint64_t p1, uint64_t nblk, uint64_t slice)
+{
+    SlicePiece r;
+    r.first = g0 <= p0 ? 0 : slice_cut(g0 - p0, nblk);
+    r.end = g1 >= p1 ? nblk : slice_cut(g1 - p0, nblk);
+    r.reporters = (g0 <= p0 && g1 >= p1) ? 1u : (uint32_t)((p1 - 1) / slice - p0 / slice) + 1u;
+    return r;
+}
+
 // Where the bytes of a segment live: flat (one offset) or through a page table.
 struct SegAddr {
     const int32_t* table;     // nullptr: flat

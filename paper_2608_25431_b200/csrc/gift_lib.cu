@@ -128,24 +128,6 @@ __device__ __forceinline__ uint64_t seg_unit(const CallArgs& a, const gift_seg& 
     return (uint64_t)(uint32_t)a.page_table[(uint64_t)s.page0 + k];
 }
 
-// Weight of a segment in the static work split (see scan_kernel).
-constexpr uint32_t SEG_WEIGHT = 64u;
-constexpr uint32_t MIN_SLICE = 256u;      // small calls: fewer warps rather than thinner slices
-
-__device__ __forceinline__ unsigned long long weight_of(uint64_t len, uint32_t st)
-{
-    if (st != 0) return 0ull;
-    return ((seg_blocks(len) + 31u) & ~(uint64_t)31u) + SEG_WEIGHT;   // an empty segment still needs its tag
-}
-
-// First block of the piece that starts at weight distance d from the segment's start.
-__device__ __forceinline__ uint64_t slice_cut(uint64_t d, uint64_t nblk)
-{
-    if (d <= SEG_WEIGHT) return 0;
-    const uint64_t b = d - SEG_WEIGHT;
-    return b >= nblk ? nblk : (b & ~(uint64_t)31u);
-}
-
 // ---------------------------------------------------------------------------
 // 1. plan: validation, label check (paper sec. 3 step 4, sec. 4.2), pre-status
 // ---------------------------------------------------------------------------
@@ -204,7 +186,7 @@ __global__ void plan_kernel(CallArgs a)
         a.status[s] = st;
         a.acc[s] = make_uint4(0u, 0u, 0u, 0u);
         a.ticket[s] = 0u;
-        a.wprefix[s] = weight_of(seg.len, st);      // the scan turns the weights into their prefix sum in place
+        a.wprefix[s] = st != 0 ? 0ull : seg_weight(seg_blocks(seg.len));      // the scan turns the weights into their prefix sum in place
         if (st != 0 && MODE == MODE_ENCRYPT) {
             reinterpret_cast<uint4*>(a.tags)[s] = make_uint4(0u, 0u, 0u, 0u);
         }
@@ -281,7 +263,7 @@ __global__ void scan_kernel(CallArgs a)
     if (tid == 0) {
         a.wprefix[a.nseg] = carry;
         unsigned long long slice = (carry + a.resident_warps - 1) / a.resident_warps;
-        if (slice < MIN_SLICE) slice = MIN_SLICE;
+        if (slice < MIN_SLICE) slice = MIN_SLICE;   // small calls: fewer warps rather than thinner slices
         a.glob->total_weight = carry;
         a.glob->slice = slice;
     }
@@ -465,10 +447,10 @@ __global__ void __launch_bounds__(THREADS, 1) crypt_kernel(const __grid_constant
         const uint64_t nblk = seg_blocks(seg.len);
         // this warp's piece of the segment, and how many warps have one (each reports once,
         // with or without blocks; the last report finishes the tag)
-        const uint64_t run_first = g0 <= p0 ? 0 : slice_cut(g0 - p0, nblk);
-        const uint64_t run_end = g1 >= p1 ? nblk : slice_cut(g1 - p0, nblk);
-        const uint32_t run_n = (uint32_t)(run_end - run_first);
-        const uint32_t seg_runs = (g0 <= p0 && g1 >= p1) ? 1u : (uint32_t)((p1 - 1) / slice - p0 / slice) + 1u;
+        const SlicePiece piece = slice_piece(g0, g1, p0, p1, nblk, slice);
+        const uint64_t run_first = piece.first;
+        const uint32_t run_n = (uint32_t)(piece.end - piece.first);
+        const uint32_t seg_runs = piece.reporters;
 
         // this warp's copy of the owner's key material (512 bytes: one uint4 per lane)
         __syncwarp();

@@ -103,6 +103,17 @@ void hc_power(const uint8_t* key, uint64_t e, uint8_t* out)
     store_block(out, o);
 }
 
+uint64_t hc_seg_weight(uint64_t nblk) { return seg_weight(nblk); }
+
+uint32_t hc_min_slice(void) { return MIN_SLICE; }
+
+// out = {first, end, reporters} of slice [g0, g1) in the segment with weight range [p0, p1)
+void hc_slice_piece(uint64_t g0, uint64_t g1, uint64_t p0, uint64_t p1, uint64_t nblk, uint64_t slice, uint64_t out[3])
+{
+    const SlicePiece r = slice_piece(g0, g1, p0, p1, nblk, slice);
+    out[0] = r.first; out[1] = r.end; out[2] = r.reporters;
+}
+
 }  // extern "C"
 
 // One whole segment, decomposed exactly as the kernel does: runs of run_blocks

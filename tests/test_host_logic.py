@@ -158,3 +158,69 @@ def test_paged_addressing_reproduces_gcm(hc, pb, chains):
         for o, l in sl:
             touched[o:o + l] = True
         assert np.array_equal(out[~touched], buf[~touched])
+
+
+def test_static_work_split_tiles_every_segment_exactly(hc):
+    """The kernel's split arithmetic, compiled for the host: for random tables and warp counts
+    the pieces of every accepted segment tile [0, nblk) in order, start on whole rows, and
+    exactly the predicted number of slices report on it (the last report finishes its tag)."""
+    hc.hc_seg_weight.restype = C.c_uint64
+    hc.hc_seg_weight.argtypes = [C.c_uint64]
+    hc.hc_min_slice.restype = C.c_uint32
+    hc.hc_slice_piece.argtypes = [C.c_uint64] * 6 + [C.c_void_p]
+    rng = np.random.default_rng(31)
+    out = np.zeros(3, dtype=np.uint64)
+
+    def check(nblks, accepted, n_warps):
+        w = np.array([hc.hc_seg_weight(int(n)) if a else 0 for n, a in zip(nblks, accepted)], dtype=np.uint64)
+        prefix = np.concatenate([[0], np.cumsum(w)]).astype(np.uint64)
+        total = int(prefix[-1])
+        slice_ = max((total + n_warps - 1) // n_warps, hc.hc_min_slice())
+        pieces = [[] for _ in nblks]
+        reports = np.zeros(len(nblks), dtype=np.int64)
+        predicted = np.zeros(len(nblks), dtype=np.int64)
+        for wi in range(n_warps):
+            g0 = wi * slice_
+            if g0 >= total:
+                break
+            g1 = min(g0 + slice_, total)
+            s = int(np.searchsorted(prefix[:-1], g0, side="right")) - 1      # largest s with prefix[s] <= g0
+            while s < len(nblks) and int(prefix[s]) < g1:
+                p0, p1 = int(prefix[s]), int(prefix[s + 1])
+                if p1 > p0:
+                    hc.hc_slice_piece(g0, g1, p0, p1, int(nblks[s]), slice_, _p(out))
+                    first, end, rep = int(out[0]), int(out[1]), int(out[2])
+                    assert first <= end <= nblks[s]
+                    assert first % 32 == 0 or first == nblks[s]
+                    if end > first:
+                        pieces[s].append((first, end))
+                    reports[s] += 1
+                    assert predicted[s] in (0, rep)
+                    predicted[s] = rep
+                s += 1
+        for s, n in enumerate(nblks):
+            if not accepted[s]:
+                assert reports[s] == 0
+                continue
+            assert reports[s] == predicted[s] >= 1, (s, reports[s], predicted[s])
+            pos = 0
+            for a, b in pieces[s]:                                             # warps visit a segment in order
+                assert a == pos
+                pos = b
+            assert pos == n
+
+    check(np.full(256, 4001), np.ones(256, bool), 3552)                        # the decode-row table
+    check(np.array([0]), np.array([True]), 3552)
+    check(np.array([5, 0, 0, 70000]), np.array([True, True, False, True]), 4)
+    for _ in range(120):
+        n = int(rng.integers(1, 300))
+        kind = int(rng.integers(0, 4))
+        if kind == 0:
+            nb = rng.integers(0, 6, size=n)
+        elif kind == 1:
+            nb = rng.integers(0, 5000, size=n)
+        elif kind == 2:
+            nb = rng.choice([0, 1, 31, 32, 33, 1024, 16384, 100000], size=n)
+        else:
+            nb = (rng.pareto(1.0, size=n) * 50).astype(np.int64)
+        check(nb.astype(np.int64), rng.random(n) < 0.9, int(rng.choice([1, 7, 3552, 4736])))
