@@ -503,7 +503,11 @@ def main():
     # ciphertext, tags and status words.  With a layer-major pool the work is cut into one
     # chunk per layer over three streams (hostio.HostExporter) so that upload, cipher and
     # download overlap; other workloads go through in one piece.
+    e2e_ready = False
     if not args.no_e2e:
+        # set-up first, then all ranks agree whether to go on: a rank that could not get its pinned
+        # buffers must not leave the others waiting at the barriers of the timed region
+        setup_error = None
         try:
             from paper_2608_25431_b200 import hostio
             h_in = torch.empty(w.buf_bytes, dtype=torch.uint8, pin_memory=True)
@@ -522,7 +526,14 @@ def main():
             if exporter is None and w.buf_bytes * 3 + (4 << 30) < torch.cuda.mem_get_info()[0]:
                 pipeline = hostio.StepPipeline(w.max_users, w.user_ids, w.keys, w.buf_bytes, nseg, local, args.flags)
                 h_out, h_tags, h_status = pipeline.h_out[0], pipeline.h_tags[0], pipeline.h_status[0]
-
+        except RuntimeError as e:
+            setup_error = str(e)[:200]
+        e2e_ready = replicas.total(0.0 if setup_error is None else 1.0, "cuda") == 0.0
+        if not e2e_ready:
+            line["e2e"] = {"value": None, "unit": UNIT,
+                           "error": setup_error or "another rank could not set up its host buffers"}
+    if e2e_ready:
+        try:
             def e2e_step():
                 if exporter is not None:
                     ctx.propagate_labels(binding.RULE_IDENTITY, [om_src], om, viol)
