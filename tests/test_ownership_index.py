@@ -65,6 +65,99 @@ def test_slice_runs_match_brute_force():
         B.slice_runs(rec, (0, 0, 0, 0, 0), (3, 1, 1, 1, 8))  # out of range
 
 
+# ---- pins of the brute-force oracle: every expected value below was worked out by hand ----
+#
+# Tensor of paper sec. 4.2's example, C[layer][block][kv][slot][dim] with shape (2, 3, 2, 16, 8) and
+# 2-byte elements.  Byte strides: dim 2, slot 16, kv 256, block 512, layer 1536; 3072 bytes in all.
+
+def test_oracle_slice_runs_hand_computed():
+    shape, elem = (2, 3, 2, 16, 8), 2
+    hand = [
+        # C[1,2,:,0:8,:]: slots 0..7 of one kv half are 8*16 = 128 contiguous bytes; the two halves start
+        # at 1536 + 2*512 + {0, 256} = 2560 and 2816, i.e. runs number 20 and 22
+        (((1, 2, 0, 0, 0), (2, 3, 2, 8, 8)), 128, [20, 22]),
+        # C[1,2,:,8:16,:]: the other eight slots, 128 bytes further on
+        (((1, 2, 0, 8, 0), (2, 3, 2, 16, 8)), 128, [21, 23]),
+        # C[:,1,:,:,:]: a whole block (512 bytes) per layer, at 512 and 1536 + 512 = 2048
+        (((0, 1, 0, 0, 0), (2, 2, 2, 16, 8)), 512, [1, 4]),
+        # C[:,:,1,4:8,:]: four slots = 64 bytes at layer*1536 + block*512 + 256 + 4*16
+        (((0, 0, 1, 4, 0), (2, 3, 2, 8, 8)), 64, [5, 13, 21, 29, 37, 45]),
+        # C[1,:,0,3,:]: single slots of 16 bytes at 1536 + block*512 + 48 = 1584, 2096, 2608
+        (((1, 0, 0, 3, 0), (2, 3, 1, 4, 8)), 16, [99, 131, 163]),
+        # the whole tensor is one run
+        (((0, 0, 0, 0, 0), (2, 3, 2, 16, 8)), 3072, [0]),
+    ]
+    rec = B.TensorRec.make(0, shape, elem, [0, 1, 3])
+    for (lo, hi), run, table in hand:
+        orun, otable = OI.slice_runs(shape, elem, lo, hi)
+        assert orun == run and otable.tolist() == table, (lo, hi)
+        crun, ctable = B.slice_runs(rec, lo, hi)                 # the library's host call agrees with the same values
+        assert crun == run and ctable.tolist() == table, (lo, hi)
+    # the byte offsets themselves for the smallest case: three rows of eight 2-byte elements
+    assert OI.slice_byte_offsets(shape, elem, (1, 0, 0, 3, 0), (2, 3, 1, 4, 8)).tolist() == \
+        list(range(1584, 1600)) + list(range(2096, 2112)) + list(range(2608, 2624))
+
+
+def test_oracle_expand_owners_hand_computed():
+    # shape (2, 3, 2, 4, 2), 2-byte elements: a slot row is 4 bytes, a kv half 16, a block 32, a layer 96.
+    # Ownership by (layer, block, slot): the three extents differ, so a transposed broadcast cannot pass.
+    shape, elem, odims = (2, 3, 2, 4, 2), 2, [0, 1, 3]
+    P, X = -1, -3                                               # PARAM, CONFLICT
+    lvl2 = [[[1, 1, 2, 2], [3, 3, 3, 3], [0, 1, 0, 1]],
+            [[4, 4, 4, 4], [P, P, 5, 5], [2, 2, 2, 2]]]
+    hand = {
+        # one label per slot row: the level-2 record, once per kv half
+        4: [1, 1, 2, 2, 1, 1, 2, 2] + [3] * 8 + [0, 1, 0, 1, 0, 1, 0, 1] +
+           [4] * 8 + [P, P, 5, 5, P, P, 5, 5] + [2] * 8,
+        # two slots per run: they agree, or the run is CONFLICT
+        8: [1, 2, 1, 2, 3, 3, 3, 3, X, X, X, X, 4, 4, 4, 4, P, 5, P, 5, 2, 2, 2, 2],
+        # a kv half (four slots) per run
+        16: [X, X, 3, 3, X, X, 4, 4, X, X, 2, 2],
+        # a whole block per run
+        32: [X, 3, X, 4, X, 2],
+        # half a slot row: part of one record, the label twice
+        2: [v for v in ([1, 1, 2, 2, 1, 1, 2, 2] + [3] * 8 + [0, 1, 0, 1, 0, 1, 0, 1] +
+                        [4] * 8 + [P, P, 5, 5, P, P, 5, 5] + [2] * 8) for _ in (0, 1)],
+    }
+    for run_bytes, want in hand.items():
+        assert OI.expand_owners(shape, elem, odims, lvl2, run_bytes).tolist() == want, run_bytes
+    # ownership by rows only (odims = (0)): every byte of a layer carries the layer's label
+    assert OI.expand_owners(shape, elem, [0], [7, 9], 48).tolist() == [7, 7, 9, 9]
+    # ownership by the innermost of the recorded dimensions only (odims = (3)): label = slot's
+    assert OI.expand_owners((1, 1, 2, 4, 2), elem, [3], [5, 6, 7, 8], 4).tolist() == [5, 6, 7, 8, 5, 6, 7, 8]
+
+
+def test_oracle_resolve_args_hand_computed():
+    OK_, UNK, SHP, ALI = 0, 1, 2, 4
+    recs = [dict(base=0x1000, shape=(4, 8), elem=2),             # 0: [0x1000, 0x1040)
+            dict(base=0x2000, shape=(4, 8), elem=2),             # 1: [0x2000, 0x2040)
+            dict(base=0x2020, shape=(16,), elem=4),              # 2: [0x2020, 0x2060)  overlaps 1 partially
+            dict(base=0x9000, shape=(2, 3, 2, 16, 8), elem=2),   # 3: [0x9000, 0x9C00)
+            dict(base=0x9010, shape=(4,), elem=4),               # 4: [0x9010, 0x9020)  inside 3
+            dict(base=0x1040, shape=(8,), elem=2)]               # 5: [0x1040, 0x1050)  touches 0, no common byte
+
+    def arg(k, group=0, shape=None):
+        return dict(base=recs[k]["base"], shape=recs[k]["shape"] if shape is None else shape, alias_group=group)
+
+    hand = [
+        ([arg(1), arg(2)], [1, 2], [ALI, ALI]),                  # partial overlap, either order
+        ([arg(2), arg(1)], [2, 1], [ALI, ALI]),
+        ([arg(3), arg(4)], [3, 4], [ALI, ALI]),                  # one inside the other, either order
+        ([arg(4), arg(3)], [4, 3], [ALI, ALI]),
+        ([arg(3, 7), arg(4, 7)], [3, 4], [OK_, OK_]),            # declared as aliases: accepted
+        ([arg(3, 7), arg(4, 8)], [3, 4], [ALI, ALI]),            # different groups: not the same declaration
+        ([arg(0), arg(5)], [0, 5], [OK_, OK_]),                  # adjacent ranges share no byte
+        ([arg(0), arg(1), arg(2), arg(5)], [0, 1, 2, 5], [OK_, ALI, ALI, OK_]),
+        ([arg(1, 0, (8, 4)), arg(2)], [1, 2], [SHP | ALI, ALI]), # wrong shape and overlapping
+        ([dict(base=0x2010, shape=(4, 8), alias_group=0), arg(2)], [-1, 2], [UNK, OK_]),   # unknown base: no record, no range
+    ]
+    for args, want_idx, want_st in hand:
+        assert OI.resolve_args(recs, args) == (want_idx, want_st), args
+        cr = [B.TensorRec.make(r["base"], r["shape"], r["elem"], [0]) for r in recs]
+        ca = [B.KernelArg.make(a["base"], a["shape"], a["alias_group"]) for a in args]
+        assert B.resolve_args(cr, ca) == (want_idx, want_st), args
+
+
 @pytest.mark.gpu
 def test_owner_expansion_and_slot_level_export_on_gpu():
     import torch
