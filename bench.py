@@ -9,7 +9,11 @@ owner's key with a per-block tag.  One step = one pass of the whole hot path ove
 batch: the four flow rules on the blocks' owner labels (copy, row-preserving, per-group
 reduction, scatter to pool pages; one fused launch), then gift_seg_encrypt (plan + label check, work split,
 CTR + GHASH, tag finish) in place.  Key
-setup is outside the step, as it is once per key change.  The path does not shard: with
+setup is outside the step, as it is once per key change.  After the timed region of the
+default workload the same step is timed on the other KV-cache configurations (config 4: 8 GiB
+of Zipf-skewed page chains; config 5: the 64 GiB mixed batch) and on the decode-step rows
+(config 2), each with its own kernel time, clock samples and roofline fraction
+(`extra.configs`).  The path does not shard: with
 --gpus N every rank runs an independent replica on its own GPU (no collective on the data
 path) and the value is the sum of the replicas over the slowest rank's time.
 """
@@ -67,7 +71,7 @@ def build_workload(name: str, layers: int):
 class ClockSampler(threading.Thread):
     """Samples SM clock, power and throttle reasons of one GPU through NVML while the timed region runs."""
 
-    def __init__(self, index: int, period: float = 0.1):
+    def __init__(self, index: int, period: float = 0.015):
         super().__init__(daemon=True)
         self.index, self.period = index, period
         self.samples, self.reasons, self.stop_flag = [], set(), threading.Event()
@@ -194,6 +198,186 @@ def workload_config(args, w):
             else "L2 flushed between iterations", "parallelism": "replicas"}
 
 
+class Bench:
+    """One workload resident on the device with everything its step needs."""
+
+    def __init__(self, name, layers, flags, local, rank):
+        import torch
+        from paper_2608_25431_b200 import binding, device_fill, workloads as W
+        self.torch, self.binding = torch, binding
+        self.name = name
+        w = build_workload(name, layers)
+        free, _ = torch.cuda.mem_get_info()
+        self.layers = layers
+        while name in ("c3", "c5") and self.layers > 1 and w.buf_bytes + (2 << 30) > free:
+            self.layers //= 2
+            w = build_workload(name, self.layers)
+        self.w = w
+        self.nseg = nseg = len(w.segs)
+        self.payload = w.payload_bytes
+        self.ctx = ctx = binding.Ctx(w.max_users, local, flags)
+        ctx.set_keys(w.user_ids, w.keys)
+        ctx.reserve(nseg)
+        self.buf = buf = torch.empty(w.buf_bytes, dtype=torch.uint8, device="cuda")
+        if w.buf is not None:
+            buf.copy_(torch.from_numpy(w.buf))
+        elif name == "c4":
+            device_fill.fill_bytes(buf, W.SEED_BASE + 4 + rank)
+        else:
+            device_fill.fill_bf16_normal(buf, W.SEED_BASE + 3 + rank, 1.0)
+        self.segs = torch.from_numpy(w.segs.view(np.uint8).copy()).cuda()
+        self.table = torch.from_numpy(w.page_table).cuda() if w.page_table is not None else None
+        self.om_src = torch.from_numpy(w.owner_map).cuda()
+        self.om = torch.empty_like(self.om_src)
+        self.viol = torch.zeros(2, dtype=torch.int32, device="cuda")
+        self.tags = torch.zeros((nseg, 16), dtype=torch.uint8, device="cuda")
+        self.status = torch.zeros(nseg, dtype=torch.int32, device="cuda")
+        self.flush = torch.empty(512 << 20, dtype=torch.uint8, device="cuda") if self.payload <= (256 << 20) else None
+        self.tables = dict(page_table=self.table, page_bytes=w.page_bytes, owner_map=self.om, unit_bytes=w.unit_bytes)
+        self._rules()
+
+    def _rules(self):
+        """Flow rules of the step.  For the KV handoff (config 3) the labels start per segment in
+        table order (layer-major, each user's blocks contiguous) and pass through all four rule
+        kinds: the copy (IDENTITY), a row-preserving kernel with a parameter operand (ROWWISE), a
+        reduction per (layer, user) over that group's blocks (SEGREDUCE) and the scatter to physical
+        pool pages through the inverse block table (BROADCAST).  The result is the page owner map
+        that the export's label check reads.  The mixed batch (config 5) runs the four rules on its
+        token owner map (copy, row-preserving, attention over each request's KV blocks, gather of
+        the request's last token) before the export checks its per-(layer, token) labels.  The
+        other workloads apply the copy rule to their unit map."""
+        torch, binding, w, ctx = self.torch, self.binding, self.w, self.ctx
+        self.rules4 = None
+        self.keep = []
+        if self.name == "c3":
+            x, nseg = w.extra, self.nseg
+            om_seg = torch.from_numpy(w.segs["owner"].astype(np.int32)).cuda()
+            tmp_a, tmp_b, tmp_c = torch.empty_like(om_seg), torch.empty_like(om_seg), torch.empty_like(om_seg)
+            param = torch.full((1,), binding.OWNER_PARAM, dtype=torch.int32, device="cuda")
+            grp = np.concatenate([[0], np.cumsum(np.tile(x["nblk"], x["layers"]))]).astype(np.int32)
+            grp_ptr = torch.from_numpy(grp).cuda()
+            src_idx = torch.arange(nseg, dtype=torch.int32, device="cuda")
+            inv = np.empty(nseg, dtype=np.int32)
+            inv[w.page_table] = np.arange(nseg, dtype=np.int32)
+            inv_table = torch.from_numpy(inv).cuda()
+            self.rules4 = [
+                {"kind": binding.RULE_IDENTITY, "in_maps": [om_seg], "out_map": tmp_a},
+                {"kind": binding.RULE_ROWWISE, "in_maps": [tmp_a, param], "out_map": tmp_b, "param_mask": 2},
+                {"kind": binding.RULE_SEGREDUCE, "in_maps": [tmp_b, tmp_b], "out_map": tmp_c, "seg_ptr": grp_ptr,
+                 "src_ptr": grp_ptr, "src_idx": src_idx},
+                {"kind": binding.RULE_BROADCAST, "in_maps": [tmp_c], "out_map": self.om, "gather": inv_table},
+            ]
+        elif self.name == "c5":
+            x = w.extra
+            t_own = torch.from_numpy(x["token_owner"]).cuda()
+            ta, tb, tc, td = (torch.empty_like(t_own) for _ in range(4))
+            par = torch.full((1,), binding.OWNER_PARAM, dtype=torch.int32, device="cuda")
+            kv_own = torch.from_numpy(x["kv_owner"]).cuda()
+            sp5, srcp5 = torch.from_numpy(x["seg_ptr"]).cuda(), torch.from_numpy(x["src_ptr"]).cuda()
+            bt5, ga5 = torch.from_numpy(x["block_table"]).cuda(), torch.from_numpy(x["gather"]).cuda()
+            self.rules4 = [
+                {"kind": binding.RULE_IDENTITY, "in_maps": [t_own], "out_map": ta},
+                {"kind": binding.RULE_ROWWISE, "in_maps": [ta, par], "out_map": tb, "param_mask": 2},
+                {"kind": binding.RULE_SEGREDUCE, "in_maps": [tb, kv_own], "out_map": tc, "seg_ptr": sp5, "src_ptr": srcp5,
+                 "src_idx": bt5},
+                {"kind": binding.RULE_BROADCAST, "in_maps": [tc], "out_map": td, "gather": ga5},
+            ]
+            self.token_maps = (t_own, td)
+            self.om.copy_(self.om_src)                    # per-(layer, token) labels of the handoff buffer
+        if self.rules4 is not None:
+            self.viol4 = torch.zeros(8, dtype=torch.int32, device="cuda")
+            self.run_rules4 = ctx.prepare_chain(self.rules4)
+
+    def rules(self):
+        if self.rules4 is not None:
+            self.run_rules4(self.viol4)                   # the four rules in one launch
+        else:
+            self.ctx.propagate_labels(self.binding.RULE_IDENTITY, [self.om_src], self.om, self.viol)
+
+    def step(self):
+        self.rules()
+        self.ctx.seg_encrypt(self.buf, self.buf, self.segs, self.nseg, self.tags, self.status, **self.tables)
+
+    def check(self):
+        torch = self.torch
+        assert not self.status.any().item() and int(self.viol[0].item()) == 0, "workload segments were rejected"
+        assert torch.equal(self.om, self.om_src), "propagated labels differ from the pool's owner map"
+        assert self.rules4 is None or not self.viol4[0::2].any().item(), "a flow rule reported a conflict"
+        if self.name == "c5":
+            assert torch.equal(self.token_maps[0], self.token_maps[1]), "token labels changed through the rules"
+
+    def timed(self, steps, warmup, barrier, sampler_index):
+        """Warm up, then time `steps` steps with CUDA events on the launching stream; returns the
+        measurements of this rank.  With inputs that fit in L2 the cache is flushed before every
+        step, outside the step's events."""
+        torch = self.torch
+        for _ in range(warmup):
+            if self.flush is not None:
+                self.flush.fill_(1)
+            self.step()
+        barrier()
+        self.check()
+        l0 = self.ctx.launch_count()
+        self.ctx.timing_enable(True)
+        sampler = ClockSampler(sampler_index)
+        sampler.start()
+        a = [torch.cuda.Event(enable_timing=True) for _ in range(steps)]
+        b = [torch.cuda.Event(enable_timing=True) for _ in range(steps)]
+        barrier()
+        for i in range(steps):
+            if self.flush is not None:
+                self.flush.fill_(1)
+            a[i].record()
+            self.step()
+            b[i].record()
+        barrier()
+        clocks = sampler.result()
+        step_ms = [a[i].elapsed_time(b[i]) for i in range(steps)]
+        # large inputs: the whole region first event to last (the steps run back to back);
+        # flushed inputs: the steps' own brackets
+        total_ms = a[0].elapsed_time(b[-1]) if self.flush is None else float(np.sum(step_ms))
+        crypt_ms, crypt_n = self.ctx.timing_read()
+        self.ctx.timing_enable(False)
+        return {"total_ms": total_ms, "step_ms": step_ms, "kernel_ms": crypt_ms / max(1, crypt_n),
+                "kernel_launches": crypt_n, "clocks": clocks, "launches": self.ctx.launch_count() - l0}
+
+    def close(self):
+        self.ctx.close()
+
+
+def roofline_of(w, kern_ms, clocks, sms, peaks):
+    """Roofline of the dominant kernel (the cipher kernel), which the integer pipes bind."""
+    payload, nseg = w.payload_bytes, len(w.segs)
+    nblk = int(((w.segs["len"].astype(np.int64) + 15) // 16).sum())
+    f_mhz = clocks["sm_mhz"] or 1965.0
+    hbm_gbs = peaks.get("hbm_gbs", 6650.0)
+    r_alu, r_mul, r_lds, r_issue = 64.0, 64.0, 32.0, 128.0        # lane-ops per SM clock, measured with the pipe probes
+    f = f_mhz * 1e6
+    t_alu = ALU_OPS_PER_BLOCK * nblk / (sms * r_alu * f)
+    t_mul = MUL_OPS_PER_BLOCK * nblk / (sms * r_mul * f)
+    t_lds = LDS_OPS_PER_BLOCK * nblk / (sms * r_lds * f)
+    t_issue = ALL_OPS_PER_BLOCK * nblk / (sms * r_issue * f)
+    t_hbm = (2.0 * payload + 56.0 * nseg) / (hbm_gbs * 1e9)
+    t_roof = max(t_alu, t_mul, t_lds, t_issue, t_hbm)
+    return {"bound": "alu", "achieved": ALU_OPS_PER_BLOCK * nblk / (kern_ms * 1e-3) / 1e12,
+            "peak": sms * r_alu * f / 1e12, "unit": "Top/s",
+            "frac": t_roof / (kern_ms * 1e-3), "traffic": NCU_DRAM_BYTES_PER_PAYLOAD_BYTE * payload,
+            "traffic_note": "bytes per launch: ncu DRAM bytes per payload byte on the 2-layer capture x this payload",
+            "kernel": "crypt_kernel", "kernel_ms": kern_ms,
+            "kernel_payload_gbs": payload / (kern_ms * 1e-3) / 1e9,
+            "hbm_achieved_gbs": 2.0 * payload / (kern_ms * 1e-3) / 1e9,
+            "hbm_frac_of_measured": 2.0 * payload / (kern_ms * 1e-3) / 1e9 / hbm_gbs,
+            "ceilings_gbs": {"alu": payload / t_alu / 1e9, "mul": payload / t_mul / 1e9,
+                             "lds": payload / t_lds / 1e9, "issue": payload / t_issue / 1e9,
+                             "hbm": payload / t_hbm / 1e9},
+            "frac_first_budget": (FIRST_ALU_OPS_PER_BLOCK * nblk / (sms * r_alu * f)) / (kern_ms * 1e-3),
+            "budget_per_block": {"alu": ALU_OPS_PER_BLOCK, "mul": MUL_OPS_PER_BLOCK, "lds": LDS_OPS_PER_BLOCK,
+                                 "all": ALL_OPS_PER_BLOCK, "first_alu": FIRST_ALU_OPS_PER_BLOCK},
+            "sm_mhz_used": f_mhz,
+            "peak_source": "148 SMs x 64 integer lanes x sampled SM clock; HBM from MEASURED_PEAKS.json (of measured)"
+            if peaks else "fallback HBM 6650 GB/s (of fallback)"}
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -202,10 +386,11 @@ def main():
     ap.add_argument("--impl", default="gift", choices=["gift", "reference"])
     ap.add_argument("--workload", default="c3", choices=["c2", "c3", "c4", "c5"])
     ap.add_argument("--layers", type=int, default=32)
-    ap.add_argument("--flags", type=lambda s: int(s, 0), default=0, help="kernel variant, see gift.h")
+    ap.add_argument("--flags", type=lambda s: int(s, 0), default=0, help="context flags, see gift.h")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-extra", action="store_true")
+    ap.add_argument("--no-configs", action="store_true", help="skip the other configurations (extra.configs)")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "gift" else args.warmup
 
@@ -215,7 +400,7 @@ def main():
 
     import torch
     import torch.distributed as dist
-    from paper_2608_25431_b200 import binding, device_fill, replicas, workloads as W
+    from paper_2608_25431_b200 import binding, hostio, replicas, workloads as W
 
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
@@ -231,153 +416,57 @@ def main():
             dist.barrier()
         torch.cuda.synchronize()
 
-    w = build_workload(args.workload, args.layers)
-    free, _ = torch.cuda.mem_get_info()
-    if w.buf_bytes + (2 << 30) > free and args.workload in ("c3", "c5"):
-        while args.layers > 1 and w.buf_bytes + (2 << 30) > free:
-            args.layers //= 2
-            w = build_workload(args.workload, args.layers)
-    nseg = len(w.segs)
-    ctx = binding.Ctx(w.max_users, local, args.flags)
-    ctx.set_keys(w.user_ids, w.keys)
-    ctx.reserve(nseg)
-    buf = torch.empty(w.buf_bytes, dtype=torch.uint8, device="cuda")
-    if w.buf is not None:
-        buf.copy_(torch.from_numpy(w.buf))
-    elif args.workload == "c4":
-        device_fill.fill_bytes(buf, W.SEED_BASE + 4 + rank)
-    else:
-        device_fill.fill_bf16_normal(buf, W.SEED_BASE + 3 + rank, 1.0)
-    segs = torch.from_numpy(w.segs.view(np.uint8).copy()).cuda()
-    table = torch.from_numpy(w.page_table).cuda() if w.page_table is not None else None
-    om_src = torch.from_numpy(w.owner_map).cuda()
-    om = torch.empty_like(om_src)
-    viol = torch.zeros(2, dtype=torch.int32, device="cuda")
-    tags = torch.zeros((nseg, 16), dtype=torch.uint8, device="cuda")
-    status = torch.zeros(nseg, dtype=torch.int32, device="cuda")
-    flush = torch.empty(512 << 20, dtype=torch.uint8, device="cuda") if w.payload_bytes <= (256 << 20) else None
-    payload = w.payload_bytes
-
-    # Flow rules of the step.  For the KV handoff the labels start per segment in table order
-    # (layer-major, each user's blocks contiguous) and pass through all four rule kinds: the
-    # copy (IDENTITY), a row-preserving kernel with a parameter operand (ROWWISE), a reduction
-    # per (layer, user) over that group's blocks (SEGREDUCE) and the scatter to physical pool
-    # pages through the inverse block table (BROADCAST).  The result is the page owner map that
-    # the export's label check reads.  Other workloads apply the copy rule to their unit map.
-    rules4 = None
-    if args.workload == "c3":
-        x = w.extra
-        om_seg = torch.from_numpy(w.segs["owner"].astype(np.int32)).cuda()
-        tmp_a, tmp_b = torch.empty_like(om_seg), torch.empty_like(om_seg)
-        param = torch.full((1,), binding.OWNER_PARAM, dtype=torch.int32, device="cuda")
-        grp = np.concatenate([[0], np.cumsum(np.tile(x["nblk"], x["layers"]))]).astype(np.int32)
-        grp_ptr = torch.from_numpy(grp).cuda()
-        src_idx = torch.arange(nseg, dtype=torch.int32, device="cuda")
-        inv = np.empty(nseg, dtype=np.int32)
-        inv[w.page_table] = np.arange(nseg, dtype=np.int32)
-        inv_table = torch.from_numpy(inv).cuda()
-        tmp_c = torch.empty_like(om_seg)
-        rules4 = [
-            {"kind": binding.RULE_IDENTITY, "in_maps": [om_seg], "out_map": tmp_a},
-            {"kind": binding.RULE_ROWWISE, "in_maps": [tmp_a, param], "out_map": tmp_b, "param_mask": 2},
-            {"kind": binding.RULE_SEGREDUCE, "in_maps": [tmp_b, tmp_b], "out_map": tmp_c, "seg_ptr": grp_ptr,
-             "src_ptr": grp_ptr, "src_idx": src_idx},
-            {"kind": binding.RULE_BROADCAST, "in_maps": [tmp_c], "out_map": om, "gather": inv_table},
-        ]
-        viol4 = torch.zeros(8, dtype=torch.int32, device="cuda")
-        run_rules4 = ctx.prepare_chain(rules4)
-
-    def step():
-        if flush is not None:
-            flush.fill_(1)
-        if rules4 is not None:
-            run_rules4(viol4)                           # the four rules in one launch
-        else:
-            ctx.propagate_labels(binding.RULE_IDENTITY, [om_src], om, viol)
-        ctx.seg_encrypt(buf, buf, segs, nseg, tags, status, page_table=table, page_bytes=w.page_bytes,
-                        owner_map=om, unit_bytes=w.unit_bytes)
-
-    for _ in range(args.warmup):
-        step()
-    barrier()
-    assert not status.any().item() and int(viol[0].item()) == 0, "workload segments were rejected"
-    assert torch.equal(om, om_src), "propagated labels differ from the pool's owner map"
-    assert rules4 is None or not viol4[0::2].any().item(), "a flow rule reported a conflict"
-    l0 = ctx.launch_count()
-    ctx.timing_enable(True)
-    sampler = ClockSampler(physical_gpu_index(local))
-    sampler.start()
-    ev = [torch.cuda.Event(enable_timing=True) for _ in range(args.steps + 1)]
-    barrier()
-    ev[0].record()
-    for i in range(args.steps):
-        step()
-        ev[i + 1].record()
-    barrier()
-    clocks = sampler.result()
-    total_ms = ev[0].elapsed_time(ev[-1])
-    step_ms = [ev[i].elapsed_time(ev[i + 1]) for i in range(args.steps)]
-    crypt_ms, crypt_n = ctx.timing_read()
-    ctx.timing_enable(False)
-    launches = ctx.launch_count() - l0 + (args.steps if flush is not None else 0) * 0
-    value, total_ms_max = replicas.job_throughput(payload * args.steps, total_ms, "cuda")
-    ms_per_step = total_ms_max / args.steps
-
-    # ---- roofline of the dominant kernel (the cipher kernel), bound by the integer pipes ----
-    nblk = int(((w.segs["len"].astype(np.int64) + 15) // 16).sum())
-    kern_ms = crypt_ms / max(1, crypt_n)
-    f_mhz = clocks["sm_mhz"] or 1965.0
     sms = torch.cuda.get_device_properties(local).multi_processor_count
     peaks = json.load(open(os.path.join(ROOT, "MEASURED_PEAKS.json"))) if os.path.exists(
         os.path.join(ROOT, "MEASURED_PEAKS.json")) else {}
-    hbm_gbs = peaks.get("hbm_gbs", 6650.0)
-    r_alu, r_mul, r_lds, r_issue = 64.0, 64.0, 32.0, 128.0        # lane-ops per SM clock, measured with gift_probe_pipe
-    f = f_mhz * 1e6
-    t_alu = ALU_OPS_PER_BLOCK * nblk / (sms * r_alu * f)
-    t_mul = MUL_OPS_PER_BLOCK * nblk / (sms * r_mul * f)
-    t_lds = LDS_OPS_PER_BLOCK * nblk / (sms * r_lds * f)
-    t_issue = ALL_OPS_PER_BLOCK * nblk / (sms * r_issue * f)
-    t_hbm = (2.0 * payload + 56.0 * nseg) / (hbm_gbs * 1e9)
-    t_roof = max(t_alu, t_mul, t_lds, t_issue, t_hbm)
-    achieved_tops = ALU_OPS_PER_BLOCK * nblk / (kern_ms * 1e-3) / 1e12
-    peak_tops = sms * r_alu * f / 1e12
-    roofline = {"bound": "alu", "achieved": achieved_tops, "peak": peak_tops, "unit": "Top/s",
-                "frac": t_roof / (kern_ms * 1e-3), "traffic": NCU_DRAM_BYTES_PER_PAYLOAD_BYTE * payload,
-                "traffic_note": "bytes per launch: ncu DRAM bytes per payload byte on the 2-layer capture x this payload",
-                "kernel": "crypt_kernel", "kernel_ms": kern_ms, "kernel_launches": crypt_n,
-                "kernel_payload_gbs": payload / (kern_ms * 1e-3) / 1e9,
-                "hbm_achieved_gbs": 2.0 * payload / (kern_ms * 1e-3) / 1e9,
-                "hbm_frac_of_measured": 2.0 * payload / (kern_ms * 1e-3) / 1e9 / hbm_gbs,
-                "ceilings_gbs": {"alu": payload / t_alu / 1e9, "mul": payload / t_mul / 1e9,
-                                 "lds": payload / t_lds / 1e9, "issue": payload / t_issue / 1e9,
-                                 "hbm": payload / t_hbm / 1e9},
-                "frac_first_budget": (FIRST_ALU_OPS_PER_BLOCK * nblk / (sms * r_alu * f)) / (kern_ms * 1e-3),
-                "budget_per_block": {"alu": ALU_OPS_PER_BLOCK, "mul": MUL_OPS_PER_BLOCK, "lds": LDS_OPS_PER_BLOCK,
-                                     "all": ALL_OPS_PER_BLOCK, "first_alu": FIRST_ALU_OPS_PER_BLOCK},
-                "sm_mhz_used": f_mhz,
-                "peak_source": "148 SMs x 64 integer lanes x sampled SM clock; HBM from MEASURED_PEAKS.json (of measured)"
-                if peaks else "fallback HBM 6650 GB/s (of fallback)"}
+    gpu_index = physical_gpu_index(local)
 
+    bench = Bench(args.workload, args.layers, args.flags, local, rank)
+    args.layers = bench.layers
+    w, ctx, nseg, payload = bench.w, bench.ctx, bench.nseg, bench.payload
+    buf, segs, table, om, om_src, viol = bench.buf, bench.segs, bench.table, bench.om, bench.om_src, bench.viol
+    tags, status = bench.tags, bench.status
+    m = bench.timed(args.steps, args.warmup, barrier, gpu_index)
+    value, total_ms_max = replicas.job_throughput(payload * args.steps, m["total_ms"], "cuda")
+    ms_per_step = total_ms_max / args.steps
+    roofline = roofline_of(w, m["kernel_ms"], m["clocks"], sms, peaks)
+    roofline["kernel_launches"] = m["kernel_launches"]
     line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
             "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
             "vs_baseline": None, "dtype": "u32", "data": "synthetic", "config": workload_config(args, w),
-            "clocks": clocks, "gpu_launches": int(launches), "roofline": roofline,
-            "step_ms_median": float(np.median(step_ms))}
+            "clocks": m["clocks"], "gpu_launches": int(m["launches"]), "roofline": roofline,
+            "step_ms_median": float(np.median(m["step_ms"]))}
+
+    def timed(fn, n=5):
+        fn()
+        torch.cuda.synchronize()
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record()
+        for _ in range(n):
+            fn()
+        b.record()
+        torch.cuda.synchronize()
+        return a.elapsed_time(b) / n
+
+    def graph_of(fn):
+        side = torch.cuda.Stream()
+        side.wait_stream(torch.cuda.current_stream())
+        with torch.cuda.stream(side):
+            fn()
+        torch.cuda.current_stream().wait_stream(side)
+        torch.cuda.synchronize()
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g):
+            fn()
+        return g
 
     # ---- other rates of the same path (not in the timed region) ----
     if not args.no_extra and rank == 0:
-        def timed(fn, n=5):
-            fn()
-            torch.cuda.synchronize()
-            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-            a.record()
-            for _ in range(n):
-                fn()
-            b.record()
-            torch.cuda.synchronize()
-            return a.elapsed_time(b) / n
         ctx.seg_encrypt(buf, buf, segs, nseg, tags, status, page_table=table, page_bytes=w.page_bytes)
+        ctx.timing_enable(True)
         ver = timed(lambda: ctx.verify_tags(buf, segs, nseg, tags, status, page_table=table, page_bytes=w.page_bytes))
+        ver_kernel_ms, ver_n = ctx.timing_read()
+        ctx.timing_enable(False)
         ok_verify = not status.any().item()
         dec = timed(lambda: (ctx.seg_encrypt(buf, buf, segs, nseg, tags, status, page_table=table, page_bytes=w.page_bytes),
                              ctx.seg_decrypt(buf, buf, segs, nseg, tags, status, page_table=table,
@@ -448,84 +537,50 @@ def main():
             ctx.propagate_labels(binding.RULE_SEGREDUCE, [tb, kv_own], tc, viol, seg_ptr=sp5, src_ptr=srcp5, src_idx=bt5)
             ctx.propagate_labels(binding.RULE_BROADCAST, [tc], t_out, viol, gather=ga5)
 
-        def graph_us(fn):
-            side = torch.cuda.Stream()
-            side.wait_stream(torch.cuda.current_stream())
-            with torch.cuda.stream(side):
-                fn()
-            torch.cuda.current_stream().wait_stream(side)
-            torch.cuda.synchronize()
-            g = torch.cuda.CUDAGraph()
-            with torch.cuda.graph(g):
-                fn()
-            return timed(g.replay, n=50) * 1e3
-
-        rules["four_separate_rules_graph_us"] = graph_us(four_separate)
-        rules["fused_chain_of_4_graph_us"] = graph_us(lambda: run_chain5(v8))
-        # a decode step's output rows (config 2: 256 rows of 64 004 B): direct calls and a replayed CUDA graph
-        w2 = W.config2()
-        c2 = binding.Ctx(w2.max_users, local, args.flags)
-        c2.set_keys(w2.user_ids, w2.keys)
-        c2.reserve(len(w2.segs))
-        b2 = torch.from_numpy(w2.buf).cuda()
-        s2 = torch.from_numpy(w2.segs.view(np.uint8).copy()).cuda()
-        o2 = torch.from_numpy(w2.owner_map).cuda()
-        tg2 = torch.zeros((len(w2.segs), 16), dtype=torch.uint8, device="cuda")
-        st2 = torch.zeros(len(w2.segs), dtype=torch.int32, device="cuda")
-
-        def rows_call():
-            c2.seg_encrypt(b2, b2, s2, len(w2.segs), tg2, st2, owner_map=o2, unit_bytes=w2.unit_bytes)
-
-        direct_ms = timed(rows_call, n=50)
-        side = torch.cuda.Stream()
-        side.wait_stream(torch.cuda.current_stream())
-        with torch.cuda.stream(side):
-            rows_call()
-        torch.cuda.current_stream().wait_stream(side)
-        torch.cuda.synchronize()
-        graph = torch.cuda.CUDAGraph()
-        with torch.cuda.graph(graph):
-            rows_call()
-        graph_ms = timed(graph.replay, n=50)
-        decode_rows = {"payload_mb": w2.payload_bytes / 1e6, "direct_us": direct_ms * 1e3, "graph_us": graph_ms * 1e3,
-                       "graph_gbs": w2.payload_bytes / graph_ms / 1e6}
-        del graph
-        c2.close()
-        line["extra"] = {"verify_gbs": payload / ver / 1e6, "verify_all_ok": bool(ok_verify), "token_mode": tok,
-                         "flow_rules": rules, "decode_rows": decode_rows,
-                         "launch_order_check": order,
+        g4 = graph_of(four_separate)
+        rules["four_separate_rules_graph_us"] = timed(g4.replay, n=50) * 1e3
+        g1 = graph_of(lambda: run_chain5(v8))
+        rules["fused_chain_of_4_graph_us"] = timed(g1.replay, n=50) * 1e3
+        del g4, g1
+        line["extra"] = {"verify_gbs": payload / ver / 1e6, "verify_all_ok": bool(ok_verify),
+                         "verify_kernel_gbs": payload / (ver_kernel_ms / max(1, ver_n)) / 1e6,
+                         "token_mode": tok, "flow_rules": rules, "launch_order_check": order,
                          "encrypt_plus_decrypt_gbs": 2 * payload / dec / 1e6,
                          "decrypt_restores_ok": bool(not status.any().item()),
                          "identity_rule_us": rule_us}
 
-    # ---- end to end from pinned host memory ----
-    # Every step uploads the whole plaintext pool from pinned host memory and downloads the
-    # ciphertext, tags and status words.  With a layer-major pool the work is cut into one
-    # chunk per layer over three streams (hostio.HostExporter) so that upload, cipher and
-    # download overlap; other workloads go through in one piece.
+    # ---- end to end from pinned host memory, through gift_export_to_host ----
+    # Every step runs the step's flow rules, uploads the whole plaintext pool from pinned host
+    # memory, encrypts and downloads ciphertext, tags and status words: one library call per
+    # step.  A layer-major pool is cut into one chunk per layer (the library overlaps upload,
+    # cipher and download on its three streams); page chains scattered over the pool go through
+    # as one chunk, two exports in flight on two streams.
     e2e_ready = False
     if not args.no_e2e:
         # set-up first, then all ranks agree whether to go on: a rank that could not get its pinned
         # buffers must not leave the others waiting at the barriers of the timed region
         setup_error = None
         try:
-            from paper_2608_25431_b200 import hostio
-            h_in = torch.empty(w.buf_bytes, dtype=torch.uint8, pin_memory=True)
-            h_out = torch.empty(w.buf_bytes, dtype=torch.uint8, pin_memory=True)
-            h_tags = torch.empty((nseg, 16), dtype=torch.uint8, pin_memory=True)
-            h_status = torch.empty(nseg, dtype=torch.int32, pin_memory=True)
-            h_in.copy_(buf)
             k = max(1, min(args.steps, 5))
-            exporter = None
+            slots = None
+            h_in = torch.empty(w.buf_bytes, dtype=torch.uint8, pin_memory=True)
+            h_in.copy_(buf)
             if args.workload == "c3":
                 n_slots = w.extra["n_slots"]
-                chunks = hostio.layer_chunks(w.extra["layers"], n_slots, n_slots * w.page_bytes)
-                exporter = hostio.HostExporter(w.max_users, w.user_ids, w.keys, local, 3, args.flags, n_slots)
-
-            pipeline = None
-            if exporter is None and w.buf_bytes * 3 + (4 << 30) < torch.cuda.mem_get_info()[0]:
-                pipeline = hostio.StepPipeline(w.max_users, w.user_ids, w.keys, w.buf_bytes, nseg, local, args.flags)
-                h_out, h_tags, h_status = pipeline.h_out[0], pipeline.h_tags[0], pipeline.h_status[0]
+                chunks = binding.Ctx.chunk_array(hostio.layer_chunks(w.extra["layers"], n_slots, n_slots * w.page_bytes))
+                mode = "one chunk per layer on the library's three streams"
+            else:
+                chunks = binding.Ctx.chunk_array(hostio.whole_buffer(w.buf_bytes, nseg))
+                mode = "one chunk"
+            if args.workload != "c3" and w.buf_bytes * 4 + (4 << 30) < torch.cuda.mem_get_info()[0]:
+                slots = hostio.ExportSlots(w.buf_bytes, nseg, 2, local)
+                h_out, h_tags, h_status = slots.h_out[0], slots.h_tags[0], slots.h_status[0]
+                mode = "whole-buffer exports, two in flight on two streams"
+            else:
+                h_out = torch.empty(w.buf_bytes, dtype=torch.uint8, pin_memory=True)
+                h_tags = torch.empty((nseg, 16), dtype=torch.uint8, pin_memory=True)
+                h_status = torch.empty(nseg, dtype=torch.int32, pin_memory=True)
+                d_cipher = torch.empty(w.buf_bytes, dtype=torch.uint8, device="cuda")
         except RuntimeError as e:
             setup_error = str(e)[:200]
         e2e_ready = replicas.total(0.0 if setup_error is None else 1.0, "cuda") == 0.0
@@ -535,73 +590,100 @@ def main():
     if e2e_ready:
         try:
             def e2e_step():
-                if exporter is not None:
-                    ctx.propagate_labels(binding.RULE_IDENTITY, [om_src], om, viol)
-                    exporter.export(h_in, h_out, buf, chunks, segs, tags, status, h_tags, h_status,
-                                    page_table=table, page_bytes=w.page_bytes, owner_map=om, unit_bytes=w.unit_bytes)
-                    return
-                if pipeline is not None:
-                    ctx.propagate_labels(binding.RULE_IDENTITY, [om_src], om, viol)
-                    pipeline.step(h_in, segs, nseg, page_table=table, page_bytes=w.page_bytes, owner_map=om,
-                                  unit_bytes=w.unit_bytes)
-                    return
-                buf.copy_(h_in, non_blocking=True)
-                ctx.propagate_labels(binding.RULE_IDENTITY, [om_src], om, viol)
-                ctx.seg_encrypt(buf, buf, segs, nseg, tags, status, page_table=table, page_bytes=w.page_bytes,
-                                owner_map=om, unit_bytes=w.unit_bytes)
-                h_out.copy_(buf, non_blocking=True)
-                h_tags.copy_(tags, non_blocking=True)
-                h_status.copy_(status, non_blocking=True)
+                bench.rules()
+                if slots is not None:
+                    slots.export(ctx, h_in, segs, nseg, chunks, **bench.tables)
+                else:
+                    ctx.export_to_host(h_in, h_out, buf, d_cipher, segs, nseg, chunks, tags, status, h_tags, h_status,
+                                       **bench.tables)
 
+            def e2e_wait():
+                if slots is not None:
+                    slots.wait()
+
+            l0 = ctx.launch_count()
             e2e_step()
-            if pipeline is not None:
-                pipeline.wait()
+            e2e_wait()
             barrier()
+            e2e_launches = ctx.launch_count() - l0
             ok_e2e = not bool(h_status.any().item())
             a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
             a.record()
             for _ in range(k):
                 e2e_step()
-            if pipeline is not None:
-                pipeline.wait()
+            e2e_wait()
             b.record()
             barrier()
             e2e_value, e2e_ms = replicas.job_throughput(payload, a.elapsed_time(b) / k, "cuda")
             line["e2e"] = {"value": e2e_value, "unit": UNIT,
                            "h2d_bytes_per_step": int(w.buf_bytes),
                            "d2h_bytes_per_step": int(w.buf_bytes + nseg * 20), "steps": k, "ms_per_step": e2e_ms,
-                           "mode": "one chunk per layer on 3 streams" if exporter is not None else
-                           ("whole-buffer steps, two in flight on two streams" if pipeline is not None else "one piece"),
-                           "all_status_clear": ok_e2e}
-            if exporter is not None:
+                           "mode": mode, "api": "gift_propagate_chain + gift_export_to_host",
+                           "launches_per_step": int(e2e_launches), "all_status_clear": ok_e2e}
+            if slots is None:
                 # the opposite direction: upload ciphertext + tags, decrypt on the device, status words back
                 om_imp = torch.empty_like(om)
-                exporter.import_(h_out, h_tags, buf, chunks, segs, tags, status, h_status, page_table=table,
-                                 page_bytes=w.page_bytes, owner_map=om_imp, unit_bytes=w.unit_bytes)
+                imp_tables = dict(bench.tables, owner_map=om_imp)
+                ctx.import_from_host(h_out, h_tags, buf, segs, nseg, chunks, tags, status, h_status, **imp_tables)
                 barrier()
                 a.record()
                 for _ in range(k):
-                    exporter.import_(h_out, h_tags, buf, chunks, segs, tags, status, h_status, page_table=table,
-                                     page_bytes=w.page_bytes, owner_map=om_imp, unit_bytes=w.unit_bytes)
+                    ctx.import_from_host(h_out, h_tags, buf, segs, nseg, chunks, tags, status, h_status, **imp_tables)
                 b.record()
                 barrier()
                 imp_value, imp_ms = replicas.job_throughput(payload, a.elapsed_time(b) / k, "cuda")
                 line["e2e"]["import"] = {"value": imp_value, "unit": UNIT, "ms_per_step": imp_ms,
                                          "h2d_bytes_per_step": int(w.buf_bytes + nseg * 16),
-                                         "d2h_bytes_per_step": int(nseg * 4),
+                                         "d2h_bytes_per_step": int(nseg * 4), "api": "gift_import_from_host",
                                          "all_status_clear": not bool(h_status.any().item()),
                                          "plaintext_restored": bool(torch.equal(buf[:1 << 20], h_in[:1 << 20].cuda()))}
-                exporter.close()
-            if pipeline is not None:
-                pipeline.close()
-            del h_in, h_out
+                del d_cipher
+            del h_in, h_out, slots
         except RuntimeError as e:
             line["e2e"] = {"value": None, "unit": UNIT, "error": str(e)[:200]}
 
-    if rank == 0 and world == 1 and not args.no_cpu_baseline:
-        line["cpu_baseline"] = cpu_sample(w, 15.0)
+    cpu_w = w
+    bench.close()
+    del bench, buf, segs, table, om, om_src, tags, status
+    torch.cuda.empty_cache()
 
-    ctx.close()
+    # ---- the same step on the other configurations (single GPU only; not part of `value`) ----
+    if world == 1 and not args.no_configs and not args.no_extra:
+        configs = {}
+        for name in ("c4", "c5", "c2"):
+            if name == args.workload:
+                continue
+            try:
+                b2 = Bench(name, 32, args.flags, local, rank)
+                steps = args.steps if name != "c2" else max(args.steps, 100)
+                m2 = b2.timed(steps, args.warmup, barrier, gpu_index)
+                r2 = roofline_of(b2.w, m2["kernel_ms"], m2["clocks"], sms, peaks)
+                entry = {"workload": "%s: %s, %d segments, %.3f GiB payload, %d users, %d layers" % (
+                             name, b2.w.name, b2.nseg, b2.payload / 2**30, len(b2.w.user_ids), b2.layers),
+                         "value": b2.payload * steps / (m2["total_ms"] * 1e-3) / 1e9, "unit": UNIT, "steps": steps,
+                         "ms_per_step": m2["total_ms"] / steps, "kernel_ms": m2["kernel_ms"],
+                         "kernel_payload_gbs": r2["kernel_payload_gbs"], "frac": r2["frac"],
+                         "frac_first_budget": r2["frac_first_budget"], "clocks": m2["clocks"],
+                         "gpu_launches": int(m2["launches"]),
+                         "l2": "inputs larger than L2" if b2.flush is None else "L2 flushed before every step, outside its events"}
+                if name == "c2":
+                    # the decode step's rows as a replayed CUDA graph (what a serving loop would do)
+                    g2 = graph_of(b2.step)
+                    entry["graph_us"] = timed(g2.replay, n=200) * 1e3
+                    entry["direct_us"] = timed(b2.step, n=200) * 1e3
+                    entry["graph_gbs"] = b2.payload / entry["graph_us"] / 1e3
+                    del g2
+                configs[name] = entry
+                b2.close()
+                del b2
+                torch.cuda.empty_cache()
+            except RuntimeError as e:
+                configs[name] = {"error": str(e)[:200]}
+        line.setdefault("extra", {})["configs"] = configs
+
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        line["cpu_baseline"] = cpu_sample(cpu_w, 15.0)
+
     if rank == 0:
         print(json.dumps(line))
     if world > 1:

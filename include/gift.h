@@ -2,7 +2,7 @@
  * libgift: per-user encryption of ownership-segmented GPU buffers, with the
  * ownership-label check and segment-level flow rules, for one NVIDIA B200.
  *
- * The library realises the data path of the paper's "encryption-as-isolation"
+ * The library realises the data path of the paper's encryption-as-isolation scheme
  * (paper sec. 3, workflow steps 0 and 3-6): every user datum that leaves the
  * protected domain is ciphertext under its owner's key, and data entering it
  * is decrypted with the key of the owner the untrusted framework claims, so a
@@ -28,7 +28,7 @@
  *    pointers; they are read during the call and need not outlive it.
  *  - A ctx must not be used from two threads, or on two streams, at once.
  *  - Ownership labels are int32: a user id >= 0, GIFT_OWNER_PARAM for model
- *    parameters (paper sec. 4.2: "a special ID for model parameters"),
+ *    parameters (paper sec. 4.2 gives parameters an owner id of their own),
  *    GIFT_OWNER_NONE for memory no record covers (sec. 4.2, unowned memory may
  *    not be read), GIFT_OWNER_CONFLICT for an output whose sources disagree.
  */
@@ -53,6 +53,7 @@ extern "C" {
 #define GIFT_ST_UNOWNED         4u   /* encrypt: a covered unit is NONE or CONFLICT */
 #define GIFT_ST_NO_KEY          8u   /* the owner has no key in the ctx */
 #define GIFT_ST_BAD_DESC       16u   /* descriptor misaligned, out of range, or reserved flags set */
+#define GIFT_ST_OVERLAP        32u   /* shares bytes with another segment of the call (only with GIFT_CTX_CHECK_OVERLAP) */
 
 #define GIFT_OWNER_PARAM     (-1)
 #define GIFT_OWNER_NONE      (-2)
@@ -64,7 +65,7 @@ extern "C" {
 typedef struct gift_ctx gift_ctx;
 
 /* One ownership segment: a contiguous same-owner region (paper sec. 4.1,
- * insight 1, and sec. 4.2 "Recording granularity").  40 bytes; a device array.
+ * insight 1, and sec. 4.2 on the granularity of records).  40 bytes; a device array.
  *   owner  the owner the caller claims for the segment (selects the key)
  *   flags  reserved, must be 0
  *   offset flat mode: byte offset of the segment in the buffer, multiple of 16
@@ -105,13 +106,26 @@ typedef struct {
 
 /* Create a context on CUDA device `device` able to hold keys for user ids
  * 0 .. max_users-1 (about 17 KiB of device memory per user: round keys and
- * powers of the hash subkey), max_users <= 2^20.  flags selects a kernel
- * variant: 0 for the default, else GIFT_CTX_FLAGS(threads, tables, chains) with
- * threads in {0, 512, 768, 1024} (cipher-kernel CTA size, 0 = default), tables
- * in {2, 4} (T-tables kept in shared memory) and chains in {1, 2} (hash chains
- * per lane; 2 needs 512 threads); every variant computes the same results.
+ * powers of the hash subkey), max_users <= 2^20.  flags is 0 or a set of
+ *   GIFT_CTX_TWO_TABLES     the cipher kernel keeps two AES tables (64 KiB of shared memory
+ *                           per SM) instead of four (128 KiB): a few per cent slower, for
+ *                           callers whose own kernels must share the SM
+ *   GIFT_CTX_CHECK_OVERLAP  every segment call first checks that the segments of its table
+ *                           occupy distinct memory (paper sec. 4.3, rule step 3; sec. 3 step 4:
+ *                           every byte has one owner).  A segment that shares a byte with
+ *                           another valid segment of the call, or that names one physical page
+ *                           twice, is refused like a bad descriptor: status GIFT_ST_OVERLAP,
+ *                           nothing of it read or written, tag zero on encrypt.  Empty segments
+ *                           and segments with a bad descriptor take no part.  Costs one more
+ *                           launch per call: all pairs for flat tables (at most 65 536
+ *                           segments, else GIFT_E_RANGE), one claim per physical page for paged
+ *                           ones.  Without the flag overlapping segments give undefined bytes.
+ *   GIFT_CTX_SPLIT_LAUNCH   never use the single-launch form that small tables take (for
+ *                           measurements; results are the same)
  * Host call; synchronises. */
-#define GIFT_CTX_FLAGS(threads, tables, chains)  ((uint32_t)((((threads) / 256) << 8) | ((tables) << 4) | (chains)))
+#define GIFT_CTX_TWO_TABLES     1u
+#define GIFT_CTX_CHECK_OVERLAP  2u
+#define GIFT_CTX_SPLIT_LAUNCH   4u
 int gift_ctx_create(gift_ctx** out, int device, uint32_t max_users, uint32_t flags);
 
 /* Zero all key material on the device and free the ctx.  Synchronises. */
@@ -140,7 +154,8 @@ int gift_clear_keys(gift_ctx* ctx, const int32_t* user_ids, uint32_t n, void* st
  * 16-byte GCM tag.  Otherwise the segment's dst bytes are left as they were,
  * its tag is 16 zero bytes and status[i] says why.  src may equal dst; bytes
  * outside all segments are never written.  Segments of one call must not
- * overlap.  buf_bytes is the size of src and of dst.  src and dst are addresses
+ * overlap (GIFT_CTX_CHECK_OVERLAP makes the call check it).  A table of at most 1024
+ * segments runs as a single kernel launch.  buf_bytes is the size of src and of dst.  src and dst are addresses
  * the device can dereference: device memory, or page-locked host memory mapped
  * into the device's address space (the boundary copy of sec. 4.5 fused into
  * the cipher: the kernel then reads or writes across the bus itself). */
@@ -157,8 +172,10 @@ int gift_seg_encrypt(gift_ctx* ctx, const void* src, void* dst, uint64_t buf_byt
  * point never does.  It calls no cudaMalloc, cudaFree or other allocating routine: its
  * scratch (work list, partial hashes, counters) is a fixed array inside the library image,
  * about 1.9 MB, which every GPU that loads the library holds until the process exits.
- *   - Arguments, results and status words are exactly those of gift_seg_encrypt; the ctx
- *     (created earlier, when allocation was still allowed) supplies the keys.
+ *   - Arguments, results and status words are exactly those of gift_seg_encrypt, bound AAD
+ *     included; the ctx (created earlier, when allocation was still allowed) supplies the
+ *     keys.  On a ctx with GIFT_CTX_CHECK_OVERLAP only flat tables are taken (the check of
+ *     paged tables needs memory that grows with the buffer): GIFT_E_INVAL otherwise.
  *   - nseg must not exceed GIFT_STATIC_MAX_SEGS (65536); a larger table is refused with
  *     GIFT_E_RANGE and nothing is launched.
  *   - The first call on a device looks up the array's device address; make that first
@@ -173,14 +190,15 @@ int gift_seg_encrypt_static(gift_ctx* ctx, const void* src, void* dst, uint64_t 
                             const gift_labels* labels, uint8_t* tags_out, uint32_t* status, void* stream);
 
 /* Bind additional authenticated data to the tags (no counterpart in the paper; the AAD of
- * SP 800-38D).  After this call gift_seg_encrypt, gift_seg_decrypt and gift_verify_tags
- * authenticate the 16 bytes aad16[16*i .. 16*i+15] (device array, 16-byte aligned, one
- * entry per segment of the call) together with segment i: a tag then also vouches for,
- * say, (owner, logical position, epoch), so that a ciphertext block presented under the
- * right key and nonce but in the wrong role fails verification.  NULL (the initial state)
- * turns binding off.  The pointer is used by the calls that follow, not copied.
- * gift_seg_encrypt_static ignores it. */
-int gift_ctx_bind_aad(gift_ctx* ctx, const uint8_t* aad16);
+ * SP 800-38D).  After this call gift_seg_encrypt, gift_seg_encrypt_static, gift_seg_decrypt,
+ * gift_verify_tags and the host-boundary calls authenticate the 16 bytes
+ * aad16[16*i .. 16*i+15] (device array of n entries, 16-byte aligned) together with segment i
+ * of the call's table: a tag then also vouches for, say, (owner, logical position, epoch), so
+ * that a ciphertext block presented under the right key and nonce but in the wrong role fails
+ * verification.  A call with more than n segments is refused with GIFT_E_RANGE.  NULL (the
+ * initial state) turns binding off.  The pointer is used by the calls that follow, not
+ * copied. */
+int gift_ctx_bind_aad(gift_ctx* ctx, const uint8_t* aad16, uint32_t n);
 
 /* Import (paper sec. 3 steps 3-4): decrypt each segment with the CLAIMED
  * owner's key after checking tags_in[i] over the received ciphertext.  On a
@@ -198,7 +216,7 @@ int gift_verify_tags(gift_ctx* ctx, const void* src, uint64_t buf_bytes, const g
                      uint32_t nseg, const gift_pages* pages, const uint8_t* tags_in,
                      uint32_t* status, void* stream);
 
-/* Token mode (paper sec. 4.5, "Token encryption"): each token is encrypted on its own
+/* Token mode (paper sec. 4.5, the paragraph on tokens): each token is encrypted on its own
  * with a block cipher, not as part of a stream, because the framework splits and appends
  * sequences; a 64-bit token is extended to 128 bits with a 64-bit nonce so that equal
  * tokens give different ciphertexts, and the end-of-sequence token gets a special
@@ -217,7 +235,7 @@ int gift_tok_encrypt(gift_ctx* ctx, const uint64_t* tokens, const uint64_t* nonc
 int gift_tok_decrypt(gift_ctx* ctx, const uint8_t* in16, const int32_t* owners, uint32_t n, uint64_t eos_token,
                      uint64_t* tokens_out, uint64_t* nonces_out, uint32_t* status, void* stream);
 
-/* A flow rule (paper sec. 4.3, "Generating IFT rules", steps 4 and 5): for
+/* A flow rule (paper sec. 4.3, rule generation, steps 4 and 5): for
  * every output unit, its non-parameter sources must share one owner, which the
  * output receives; operands declared as parameters must be labelled PARAM.
  * The join treats PARAM as neutral, equal users as that user, and anything
@@ -236,9 +254,11 @@ int gift_tok_decrypt(gift_ctx* ctx, const uint8_t* in16, const int32_t* owners, 
  *                        segment covers are CONFLICT
  *   GIFT_RULE_BROADCAST  out[j] = in0[gather[j]]; out-of-range gather gives CONFLICT
  * n_in is the number of input maps (ROWWISE: 1..8; SEGREDUCE: 2; others: 1),
- * n_in0 the length of in0 (BROADCAST) and n_in1 the length of in1 (SEGREDUCE).
- * All index arrays are device arrays.  seg_ptr must be non-decreasing with
- * seg_ptr[n_seg] <= n_out. */
+ * n_in0 the length of in0 (BROADCAST), n_in1 the length of in1 and n_src the length of
+ * src_idx (SEGREDUCE).  All index arrays are device arrays supplied by the untrusted
+ * framework, so nothing in them is trusted: seg_ptr and src_ptr (n_seg + 1 entries each)
+ * must be valid CSR pointers (first entry >= 0, non-decreasing, last entry <= n_out and
+ * <= n_src); if they are not, the launch as a whole is rejected: every out[j] is CONFLICT. */
 #define GIFT_RULE_IDENTITY   0u
 #define GIFT_RULE_ROWWISE    1u
 #define GIFT_RULE_SEGREDUCE  2u
@@ -251,6 +271,7 @@ typedef struct {
     uint32_t n_seg;
     uint32_t n_in0;
     uint32_t n_in1;
+    uint32_t n_src;
     const int32_t* seg_ptr;
     const int32_t* src_ptr;
     const int32_t* src_idx;
@@ -277,13 +298,14 @@ int gift_propagate_labels(gift_ctx* ctx, const gift_rule* rule, const int32_t* c
  * GIFT_E_RANGE.  Unlike gift_propagate_labels the chain takes no snapshot: a rule's output
  * must not overlap the map it gathers from (BROADCAST in0, SEGREDUCE in1), else
  * GIFT_E_INVAL; writing a map in place at the same index (IDENTITY, ROWWISE, SEGREDUCE
- * in0) is fine.  One launch of a single 8-CTA cluster: meant for maps of up to a few
- * million units. */
+ * in0) is fine; the index arrays must not be outputs of the chain.  One launch of a single
+ * thread-block cluster (16 CTAs where the device can co-schedule them, else 8): meant for
+ * maps of up to a few million units. */
 #define GIFT_CHAIN_MAX 8u
 int gift_propagate_chain(gift_ctx* ctx, const gift_rule* rules, const int32_t* const* const* in_owner_maps,
                          int32_t* const* out_owner_maps, uint32_t n_rules, uint32_t* viol, void* stream);
 
-/* Multi-stream launch-order check (paper sec. 4.4, "Concurrency control"): the ownership
+/* Multi-stream launch-order check (paper sec. 4.4, concurrency control): the ownership
  * record of a segment is extended with its last writer kernel and last reader kernels, each
  * a (stream, sequence) pair, and a kernel counts as completed once a synchronisation of its
  * stream follows its launch.  A reader of M may launch only if M's last writer, when on
@@ -313,7 +335,7 @@ typedef struct {
 int gift_check_launch_order(gift_ctx* ctx, const gift_trace* trace, uint32_t* flags, uint32_t* summary,
                             void* stream);
 
-/* Two-level ownership index (paper sec. 4.2, "Ownership data structure"): the first level
+/* Two-level ownership index (paper sec. 4.2, the ownership data structure): the first level
  * maps a base address to a tensor record (base address, shape, element size and the
  * ownership-related dimensions, e.g. (0) for the rows of a matrix or (0,1,3) of a
  * 5-dimensional KV tensor); the second level maps the subscripts of those dimensions to an
@@ -329,7 +351,7 @@ typedef struct {
 } gift_tensor_rec;
 
 /* One tensor argument of a kernel launch as the framework presents it.  Arguments that
- * carry the same non-zero alias_group are meant to alias (paper Fig. 6, "Alias" nodes). */
+ * carry the same non-zero alias_group are meant to alias (the alias nodes of the paper's flow-graph figure). */
 typedef struct {
     uint64_t base;
     uint32_t ndim, alias_group;
@@ -365,8 +387,8 @@ int gift_expand_owners(gift_ctx* ctx, const gift_tensor_rec* rec, uint64_t run_b
                        uint32_t n_units, void* stream);
 
 /* Secure swap space (paper sec. 4.5): KV blocks swapped into the monitor's own memory need
- * no encryption, but the monitor "tracks ownership of swapped KV blocks" and restores the
- * records when the blocks come back.  swap_out saves the labels of the listed units
+ * no encryption, but their ownership records must survive the round trip.  swap_out saves
+ * the labels of the listed units
  * (saved[i] = owner_map[units[i]]) and marks the units GIFT_OWNER_NONE, so that the freed
  * slots cannot be read; swap_in writes the saved labels to the units the blocks return to,
  * which need not be the ones they left.  A unit index out of range, or a swap-in onto a
@@ -395,15 +417,45 @@ uint64_t gift_launch_count(const gift_ctx* ctx);
 int gift_timing_enable(gift_ctx* ctx, int on);
 int gift_timing_read(gift_ctx* ctx, double* total_ms, uint32_t* launches);
 
-/* Issue-rate probe (diagnostics; no paper counterpart): runs a long chain of one
- * instruction kind on every SM of `device` and reports lane-operations per SM clock and
- * the SM clock seen.  kind: 0 three-input logic, 1 32x32+64 wide multiply-add, 2 byte
- * permute, 3 conflict-free shared-memory load, 4 funnel shift, 5 integer add, 6 logic and
- * wide multiply interleaved, 7 32-bit multiply-add, 8 logic and shared loads interleaved,
- * 9-19 further kinds and pairings, 20-32 instruction mixes like the cipher kernel's (wide multiply without accumulate, logic with 32-bit multiply-add,
- * with add, with permute, permute or shared load with wide multiply, and so on).
- * Host call; allocates a few KB, synchronises. */
-int gift_probe_pipe(int device, int kind, uint32_t iters, double* lane_ops_per_clk_per_sm, double* sm_mhz);
+/* Host-boundary calls (paper sec. 4.5, the swap path of KV blocks, and sec. 5, the bounce
+ * copy between host and device): export to, and import from, page-locked HOST memory with
+ * the copies fused into the call.  The table is cut into chunks (HOST array): chunk k holds
+ * the segments [seg_lo, seg_hi) of the table, all of whose bytes lie in the byte range
+ * [byte_lo, byte_hi) of the buffer; chunks must not share segments or bytes.  Chunk k runs on
+ * one of three streams the ctx owns, each with its own scratch, so that the upload of one
+ * chunk, the cipher of the previous one and the download of the one before overlap and both
+ * bus directions stay busy.  The work is ordered after what `stream` holds at the time of
+ * the call, and `stream` waits for all of it; the call itself returns without waiting.
+ * Copies are plain cudaMemcpyAsync, one per chunk and direction.  byte_lo and byte_hi are
+ * multiples of 16. */
+typedef struct {
+    uint64_t byte_lo, byte_hi;
+    uint32_t seg_lo, seg_hi;
+} gift_chunk;
+
+/* Export.  Per chunk: upload h_src[byte range] into d_plain (skipped when h_src is NULL: the
+ * plaintext is already in d_plain), clear d_cipher[byte range], encrypt the chunk's segments
+ * out of place from d_plain into d_cipher exactly as gift_seg_encrypt would (labels, status
+ * words, tags), download d_cipher[byte range] to h_dst, the chunk's tags to h_tags and its
+ * status words to h_status.  Only ciphertext leaves the device: bytes of the range that no
+ * accepted segment covers, a refused segment's bytes among them, arrive in h_dst as zeros.
+ * d_plain is left unchanged.  h_src (or NULL), h_dst, h_tags (nseg x 16) and h_status (nseg)
+ * are page-locked host memory; d_plain, d_cipher (buf_bytes each, distinct), segs, d_tags,
+ * d_status are device memory.  GIFT_E_INVAL if a chunk is out of range or empty of order
+ * (seg_lo > seg_hi, byte_lo > byte_hi). */
+int gift_export_to_host(gift_ctx* ctx, const void* h_src, void* h_dst, void* d_plain, void* d_cipher,
+                        uint64_t buf_bytes, const gift_seg* segs, uint32_t nseg, const gift_chunk* chunks,
+                        uint32_t n_chunks, const gift_pages* pages, const gift_labels* labels, uint8_t* d_tags,
+                        uint32_t* d_status, uint8_t* h_tags, uint32_t* h_status, void* stream);
+
+/* Import.  Per chunk: upload the ciphertext h_src[byte range] into d_buf and the chunk's
+ * tags from h_tags into d_tags, decrypt in place exactly as gift_seg_decrypt would (failed
+ * segments zero-filled, labels written), download the chunk's status words to h_status.  The
+ * plaintext stays on the device. */
+int gift_import_from_host(gift_ctx* ctx, const void* h_src, const uint8_t* h_tags, void* d_buf, uint64_t buf_bytes,
+                          const gift_seg* segs, uint32_t nseg, const gift_chunk* chunks, uint32_t n_chunks,
+                          const gift_pages* pages, gift_labels* labels, uint8_t* d_tags, uint32_t* d_status,
+                          uint32_t* h_status, void* stream);
 
 #ifdef __cplusplus
 }

@@ -142,8 +142,48 @@ def _aad(aad, n):
     return a
 
 
+def overlapping(segs, buf_bytes, page_table=None, page_bytes=0, owner_map=None, unit_bytes=0):
+    """uint8[nseg]: 1 where a segment shares a byte with another segment of the table, or holds one
+    byte of the buffer twice (paper sec. 4.3 rule step 3: distinct memory; sec. 3 step 4: one owner
+    per byte).  Written out from the definition: count, for every byte of the buffer, how many
+    times the valid segments of the table cover it; a segment overlaps when one of its bytes is
+    covered more than once.  Segments with an invalid descriptor and empty segments take no part."""
+    segs = np.ascontiguousarray(segs)
+    n = segs.size
+    pt, npg, om, nu = _tables(page_table, page_bytes, owner_map, unit_bytes)
+    bad = np.zeros(max(n, 1), dtype=np.uint8)
+    f = lib().gift_oracle_seg_bad_desc
+    f.restype = C.c_int
+    rc = f(C.c_uint64(buf_bytes), _p(segs), C.c_uint32(n), _p(pt) if pt is not None else None, C.c_uint32(npg),
+           C.c_uint64(page_bytes), C.c_int(1 if om is not None else 0), C.c_uint32(nu), C.c_uint64(unit_bytes), _p(bad))
+    if rc != 0:
+        raise ValueError("oracle overlapping: bad call (%d)" % rc)
+
+    def pieces(i):
+        """(start, stop) byte ranges of segment i in the buffer."""
+        ln = int(segs["len"][i])
+        if pt is None:
+            return [(int(segs["offset"][i]), int(segs["offset"][i]) + ln)]
+        out = []
+        for k in range(0, ln, page_bytes):
+            base = int(pt[int(segs["page0"][i]) + k // page_bytes]) * page_bytes
+            out.append((base, base + min(page_bytes, ln - k)))
+        return out
+
+    cover = np.zeros(buf_bytes, dtype=np.uint16)
+    for i in range(n):
+        if not bad[i]:
+            for a, b in pieces(i):
+                cover[a:b] += 1
+    flags = np.zeros(n, dtype=np.uint8)
+    for i in range(n):
+        if not bad[i] and any((cover[a:b] > 1).any() for a, b in pieces(i)):
+            flags[i] = 1
+    return flags
+
+
 def seg_encrypt(src, dst, segs, user_ids, keys, max_users, page_table=None, page_bytes=0,
-                owner_map=None, unit_bytes=0, aad=None):
+                owner_map=None, unit_bytes=0, aad=None, check_overlap=False):
     """Encrypt every segment of `segs` from src into dst (may be the same array).
 
     Returns (tags uint8[nseg,16], status uint32[nseg]).
@@ -156,20 +196,21 @@ def seg_encrypt(src, dst, segs, user_ids, keys, max_users, page_table=None, page
     n = segs.size
     tags = np.zeros((max(n, 1), 16), dtype=np.uint8)
     status = np.zeros(max(n, 1), dtype=np.uint32)
+    ovl = overlapping(segs, src.size, page_table, page_bytes, owner_map, unit_bytes) if check_overlap and n else None
     f = lib().gift_oracle_seg_encrypt
     f.restype = C.c_int
     rc = f(_p(src), _p(dst), C.c_uint64(src.size), _p(segs), C.c_uint32(n),
            _p(pt) if pt is not None else None, C.c_uint32(npg), C.c_uint64(page_bytes),
            _p(om) if om is not None else None, C.c_uint32(nu), C.c_uint64(unit_bytes),
            _p(tab), _p(has), C.c_uint32(max_users), _p(tags), _p(status),
-           _p(_aad(aad, n)) if aad is not None else None)
+           _p(_aad(aad, n)) if aad is not None else None, _p(ovl) if ovl is not None else None)
     if rc != 0:
         raise ValueError("oracle seg_encrypt: bad call (%d)" % rc)
     return tags[:n], status[:n]
 
 
 def seg_decrypt(src, dst, segs, tags, user_ids, keys, max_users, page_table=None, page_bytes=0,
-                owner_map=None, unit_bytes=0, verify_only=False, aad=None):
+                owner_map=None, unit_bytes=0, verify_only=False, aad=None, check_overlap=False):
     """Decrypt (or only verify) every segment; owner_map, when given, is updated in place.
 
     Returns status uint32[nseg].
@@ -185,13 +226,14 @@ def seg_decrypt(src, dst, segs, tags, user_ids, keys, max_users, page_table=None
     if tg.size == 0:
         tg = np.zeros(16, dtype=np.uint8)
     status = np.zeros(max(n, 1), dtype=np.uint32)
+    ovl = overlapping(segs, src.size, page_table, page_bytes, owner_map, unit_bytes) if check_overlap and n else None
     f = lib().gift_oracle_seg_decrypt
     f.restype = C.c_int
     rc = f(_p(src), _p(dst), C.c_uint64(src.size), _p(segs), C.c_uint32(n),
            _p(pt) if pt is not None else None, C.c_uint32(npg), C.c_uint64(page_bytes),
            _p(om) if om is not None else None, C.c_uint32(nu), C.c_uint64(unit_bytes),
            _p(tab), _p(has), C.c_uint32(max_users), _p(tg), _p(status), C.c_int(1 if verify_only else 0),
-           _p(_aad(aad, n)) if aad is not None else None)
+           _p(_aad(aad, n)) if aad is not None else None, _p(ovl) if ovl is not None else None)
     if rc != 0:
         raise ValueError("oracle seg_decrypt: bad call (%d)" % rc)
     return status[:n]

@@ -372,7 +372,8 @@ typedef struct {
 } oracle_seg;
 
 enum {
-    ST_TAG_MISMATCH = 1, ST_OWNER_MISMATCH = 2, ST_UNOWNED = 4, ST_NO_KEY = 8, ST_BAD_DESC = 16
+    ST_TAG_MISMATCH = 1, ST_OWNER_MISMATCH = 2, ST_UNOWNED = 4, ST_NO_KEY = 8, ST_BAD_DESC = 16,
+    ST_OVERLAP = 32
 };
 enum { OWNER_PARAM = -1, OWNER_NONE = -2, OWNER_CONFLICT = -3 };
 
@@ -463,6 +464,20 @@ static int env_bad(const seg_env* e)
     return 0;
 }
 
+/* bad[i] = 1 where segment i has an invalid descriptor (used by the overlap definition,
+ * which leaves such segments out). */
+int gift_oracle_seg_bad_desc(uint64_t buf_bytes, const oracle_seg* segs, uint32_t nseg,
+                             const int32_t* page_table, uint32_t n_pages, uint64_t page_bytes,
+                             int has_labels, uint32_t n_units, uint64_t unit_bytes, uint8_t* bad)
+{
+    static int32_t dummy;
+    seg_env e = { NULL, NULL, buf_bytes, page_table, n_pages, page_bytes,
+                  has_labels ? &dummy : NULL, n_units, unit_bytes, NULL, NULL, 0 };
+    if (env_bad(&e)) return -1;
+    for (uint32_t i = 0; i < nseg; i++) bad[i] = (uint8_t)seg_bad_desc(&e, &segs[i]);
+    return 0;
+}
+
 /* Export (paper sec. 3 steps 5-6, sec. 4.1 on key selection from the
  * ownership state): a segment is encrypted only if every unit it covers is
  * owned by the claimed owner, who must have a key.  Otherwise its destination
@@ -474,7 +489,8 @@ int gift_oracle_seg_encrypt(const uint8_t* src, uint8_t* dst, uint64_t buf_bytes
                             const int32_t* page_table, uint32_t n_pages, uint64_t page_bytes,
                             const int32_t* owner_map, uint32_t n_units, uint64_t unit_bytes,
                             const uint8_t* keys, const uint8_t* has_key, uint32_t max_users,
-                            uint8_t* tags_out, uint32_t* status, const uint8_t* aad16)
+                            uint8_t* tags_out, uint32_t* status, const uint8_t* aad16,
+                            const uint8_t* overlap)
 {
     seg_env e = { src, dst, buf_bytes, page_table, n_pages, page_bytes,
                   (int32_t*)owner_map, n_units, unit_bytes, keys, has_key, max_users };
@@ -487,6 +503,7 @@ int gift_oracle_seg_encrypt(const uint8_t* src, uint8_t* dst, uint64_t buf_bytes
         uint32_t st = 0;
         memset(tags_out + 16 * i, 0, 16);
         if (seg_bad_desc(&e, s)) { status[i] = ST_BAD_DESC; continue; }
+        if (overlap != NULL && overlap[i]) { status[i] = ST_OVERLAP; continue; }   /* refused like a bad descriptor */
         if (owner_map != NULL) {
             uint64_t nu = seg_unit_count(&e, s);
             for (uint64_t k = 0; k < nu; k++) {
@@ -521,7 +538,8 @@ int gift_oracle_seg_decrypt(const uint8_t* src, uint8_t* dst, uint64_t buf_bytes
                             const int32_t* page_table, uint32_t n_pages, uint64_t page_bytes,
                             int32_t* owner_map, uint32_t n_units, uint64_t unit_bytes,
                             const uint8_t* keys, const uint8_t* has_key, uint32_t max_users,
-                            const uint8_t* tags_in, uint32_t* status, int mode, const uint8_t* aad16)
+                            const uint8_t* tags_in, uint32_t* status, int mode, const uint8_t* aad16,
+                            const uint8_t* overlap)
 {
     seg_env e = { src, dst, buf_bytes, page_table, n_pages, page_bytes,
                   owner_map, n_units, unit_bytes, keys, has_key, max_users };
@@ -532,6 +550,7 @@ int gift_oracle_seg_decrypt(const uint8_t* src, uint8_t* dst, uint64_t buf_bytes
     for (int64_t i = 0; i < (int64_t)nseg; i++) {
         const oracle_seg* s = &segs[i];
         if (seg_bad_desc(&e, s)) { status[i] = ST_BAD_DESC; continue; }
+        if (overlap != NULL && overlap[i]) { status[i] = ST_OVERLAP; continue; }
         if (!seg_has_key(&e, s->owner)) {
             status[i] = ST_NO_KEY;
             if (mode == 0) {
@@ -558,7 +577,7 @@ int gift_oracle_seg_decrypt(const uint8_t* src, uint8_t* dst, uint64_t buf_bytes
         for (int pass = 0; pass < 2; pass++) {
             for (uint32_t i = 0; i < nseg; i++) {
                 const oracle_seg* s = &segs[i];
-                if (status[i] == ST_BAD_DESC) continue;
+                if (status[i] == ST_BAD_DESC || status[i] == ST_OVERLAP) continue;
                 int ok = status[i] == 0;
                 if ((pass == 0) != ok) continue;
                 uint64_t nu = seg_unit_count(&e, s);

@@ -43,6 +43,17 @@ def _viol(out: np.ndarray) -> np.ndarray:
     return np.array([bad.size, bad[0] if bad.size else 0xFFFFFFFF], dtype=np.uint32)
 
 
+def csr_ok(ptr, limit: int) -> bool:
+    """ptr[0] >= 0, ptr non-decreasing, ptr[-1] <= limit."""
+    p = [int(x) for x in ptr]
+    if len(p) == 0 or p[0] < 0 or p[-1] > limit:
+        return False
+    for k in range(1, len(p)):
+        if p[k] < p[k - 1]:
+            return False
+    return True
+
+
 def propagate(kind: int, inputs, n_out: int, *, param_mask: int = 0, seg_ptr=None, src_ptr=None,
               src_idx=None, gather=None):
     """Apply one flow rule; returns (out int32[n_out], viol uint32[2] = count, first index)."""
@@ -63,6 +74,12 @@ def propagate(kind: int, inputs, n_out: int, *, param_mask: int = 0, seg_ptr=Non
         # decoding-stage attention: the outputs of request s depend on its own rows and on
         # every KV block its block table names (paper sec. 7.2: the rule walks each block)
         out[:] = CONFLICT
+        # The index arrays come from the untrusted framework (paper sec. 4.3: the rule checks the
+        # arguments of the launch it is given).  Reading taken: a table that is not a valid CSR
+        # description (a pointer array that is negative, decreasing, or that runs past what it
+        # indexes) rejects the launch as a whole, i.e. every output is CONFLICT.
+        if not (csr_ok(seg_ptr, n_out) and csr_ok(src_ptr, len(src_idx))):
+            return out, _viol(out)
         covered = np.zeros(n_out, dtype=bool)
         for s in range(len(seg_ptr) - 1):
             srcs = [ins[0][t] for t in range(seg_ptr[s], seg_ptr[s + 1])]

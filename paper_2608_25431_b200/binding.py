@@ -16,7 +16,8 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.environ.get("GIFT_LIB", os.path.join(_HERE, "libgift.so"))
 
 OK, E_INVAL, E_NOMEM, E_CUDA, E_RANGE, E_ALIGN = 0, -1, -2, -3, -4, -5
-ST_TAG_MISMATCH, ST_OWNER_MISMATCH, ST_UNOWNED, ST_NO_KEY, ST_BAD_DESC = 1, 2, 4, 8, 16
+ST_TAG_MISMATCH, ST_OWNER_MISMATCH, ST_UNOWNED, ST_NO_KEY, ST_BAD_DESC, ST_OVERLAP = 1, 2, 4, 8, 16, 32
+CTX_TWO_TABLES, CTX_CHECK_OVERLAP, CTX_SPLIT_LAUNCH = 1, 2, 4
 OWNER_PARAM, OWNER_NONE, OWNER_CONFLICT = -1, -2, -3
 RULE_IDENTITY, RULE_ROWWISE, RULE_SEGREDUCE, RULE_BROADCAST = 0, 1, 2, 3
 STATIC_MAX_SEGS = 65536
@@ -27,7 +28,7 @@ EXPORTS = [
     "gift_propagate_labels", "gift_propagate_chain", "gift_tok_encrypt", "gift_tok_decrypt", "gift_check_launch_order",
     "gift_resolve_args", "gift_slice_runs", "gift_expand_owners", "gift_labels_swap_out", "gift_labels_swap_in",
     "gift_strerror", "gift_version", "gift_launch_count", "gift_timing_enable", "gift_timing_read",
-    "gift_probe_pipe",
+    "gift_export_to_host", "gift_import_from_host",
 ]
 
 
@@ -47,9 +48,14 @@ class _Labels(C.Structure):
 
 class _Rule(C.Structure):
     _fields_ = [("kind", C.c_uint32), ("n_out", C.c_uint32), ("n_in", C.c_uint32), ("n_seg", C.c_uint32),
-                ("n_in0", C.c_uint32), ("n_in1", C.c_uint32),
+                ("n_in0", C.c_uint32), ("n_in1", C.c_uint32), ("n_src", C.c_uint32),
                 ("seg_ptr", C.c_void_p), ("src_ptr", C.c_void_p), ("src_idx", C.c_void_p),
                 ("gather", C.c_void_p), ("param_mask", C.c_uint32)]
+
+
+class Chunk(C.Structure):
+    """gift_chunk: the segments [seg_lo, seg_hi) of the table and the byte range that holds them."""
+    _fields_ = [("byte_lo", C.c_uint64), ("byte_hi", C.c_uint64), ("seg_lo", C.c_uint32), ("seg_hi", C.c_uint32)]
 
 
 class _Trace(C.Structure):
@@ -155,7 +161,13 @@ def lib():
         l.gift_launch_count.argtypes = [C.c_void_p]
         l.gift_timing_enable.argtypes = [C.c_void_p, C.c_int]
         l.gift_timing_read.argtypes = [C.c_void_p, C.POINTER(C.c_double), C.POINTER(C.c_uint32)]
-        l.gift_probe_pipe.argtypes = [C.c_int, C.c_int, C.c_uint32, C.POINTER(C.c_double), C.POINTER(C.c_double)]
+        l.gift_ctx_bind_aad.argtypes = [C.c_void_p, C.c_void_p, C.c_uint32]
+        l.gift_export_to_host.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_uint64,
+                                          C.c_void_p, C.c_uint32, C.c_void_p, C.c_uint32, C.POINTER(_Pages),
+                                          C.POINTER(_Labels), C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]
+        l.gift_import_from_host.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_uint64, C.c_void_p,
+                                            C.c_uint32, C.c_void_p, C.c_uint32, C.POINTER(_Pages), C.POINTER(_Labels),
+                                            C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]
         _lib = l
     return _lib
 
@@ -220,11 +232,10 @@ class Ctx:
         self.close()
 
     def bind_aad(self, aad16):
-        """aad16: CUDA uint8 tensor [nseg, 16] authenticated with the segments of the calls that follow, or None."""
-        f = lib().gift_ctx_bind_aad
-        f.argtypes = [C.c_void_p, C.c_void_p]
+        """aad16: CUDA uint8 tensor [n, 16] authenticated with the segments of the calls that follow, or None."""
         self._aad = aad16            # keep the tensor alive while it is bound
-        _check(f(self._h, _dev(aad16)), "gift_ctx_bind_aad")
+        n = 0 if aad16 is None else aad16.numel() // 16
+        _check(lib().gift_ctx_bind_aad(self._h, _dev(aad16), n), "gift_ctx_bind_aad")
 
     def reserve(self, max_segs: int):
         _check(lib().gift_ctx_reserve(self._h, max_segs), "gift_ctx_reserve")
@@ -290,6 +301,7 @@ class Ctx:
         n_seg = seg_ptr.numel() - 1 if seg_ptr is not None else 0
         rule = _Rule(kind, n_out, len(in_maps), n_seg,
                      in_maps[0].numel(), in_maps[1].numel() if len(in_maps) > 1 else 0,
+                     src_idx.numel() if src_idx is not None else 0,
                      seg_ptr.data_ptr() if seg_ptr is not None else None,
                      src_ptr.data_ptr() if src_ptr is not None else None,
                      src_idx.data_ptr() if src_idx is not None else None,
@@ -315,6 +327,7 @@ class Ctx:
             n_out = r.get("n_out", out_map.numel())
             arr[k] = _Rule(r["kind"], n_out, len(in_maps), seg_ptr.numel() - 1 if seg_ptr is not None else 0,
                            in_maps[0].numel(), in_maps[1].numel() if len(in_maps) > 1 else 0,
+                           src_idx.numel() if src_idx is not None else 0,
                            seg_ptr.data_ptr() if seg_ptr is not None else None,
                            src_ptr.data_ptr() if src_ptr is not None else None,
                            src_idx.data_ptr() if src_idx is not None else None,
@@ -372,6 +385,36 @@ class Ctx:
         _check(f(self._h, _dev(owner_map), owner_map.numel(), _dev(units), units.numel(), _dev(saved), _dev(viol),
                  _stream_ptr(stream)), "gift_labels_swap_in")
 
+    @staticmethod
+    def chunk_array(chunks):
+        """HOST array of gift_chunk from (byte_lo, byte_hi, seg_lo, seg_hi) tuples or Chunk objects."""
+        arr = (Chunk * max(1, len(chunks)))()
+        for k, ch in enumerate(chunks):
+            arr[k] = ch if isinstance(ch, Chunk) else Chunk(*[int(v) for v in ch])
+        return arr
+
+    def export_to_host(self, h_src, h_dst, d_plain, d_cipher, segs, nseg, chunks, d_tags, d_status, h_tags, h_status,
+                       page_table=None, page_bytes=0, owner_map=None, unit_bytes=0, stream=None):
+        """gift_export_to_host; chunks is a list of (byte_lo, byte_hi, seg_lo, seg_hi) or a prepared chunk_array."""
+        arr = chunks if isinstance(chunks, C.Array) else self.chunk_array(chunks)
+        pg, lb = self._tables(page_table, page_bytes, owner_map, unit_bytes)
+        _check(lib().gift_export_to_host(self._h, _dev(h_src), _dev(h_dst), _dev(d_plain), _dev(d_cipher),
+                                         d_plain.numel() * d_plain.element_size(), _dev(segs), nseg, arr, len(arr) if len(chunks) else 0,
+                                         C.byref(pg) if pg else None, C.byref(lb) if lb else None, _dev(d_tags),
+                                         _dev(d_status), _dev(h_tags), _dev(h_status), _stream_ptr(stream)),
+               "gift_export_to_host")
+
+    def import_from_host(self, h_src, h_tags, d_buf, segs, nseg, chunks, d_tags, d_status, h_status,
+                         page_table=None, page_bytes=0, owner_map=None, unit_bytes=0, stream=None):
+        """gift_import_from_host; chunks as for export_to_host."""
+        arr = chunks if isinstance(chunks, C.Array) else self.chunk_array(chunks)
+        pg, lb = self._tables(page_table, page_bytes, owner_map, unit_bytes)
+        _check(lib().gift_import_from_host(self._h, _dev(h_src), _dev(h_tags), _dev(d_buf),
+                                           d_buf.numel() * d_buf.element_size(), _dev(segs), nseg, arr,
+                                           len(arr) if len(chunks) else 0, C.byref(pg) if pg else None,
+                                           C.byref(lb) if lb else None, _dev(d_tags), _dev(d_status), _dev(h_status),
+                                           _stream_ptr(stream)), "gift_import_from_host")
+
     def launch_count(self) -> int:
         return int(lib().gift_launch_count(self._h))
 
@@ -397,9 +440,16 @@ PROBE_KINDS = {0: "lop3", 1: "mad.wide.u32", 2: "prmt", 3: "ld.shared.u32", 4: "
 
 
 def probe_pipe(kind: int, iters: int = 2000, device: int = 0):
-    """(lane-operations per SM clock, SM MHz seen) for one instruction kind."""
+    """(lane-operations per SM clock, SM MHz seen) for one instruction kind.
+
+    Diagnostics: calls libgift_probe.so (built by build.build_probe), which is not part of libgift.so."""
+    from . import build
+    probe = C.CDLL(build.build_probe())
+    probe.gift_probe_pipe.argtypes = [C.c_int, C.c_int, C.c_uint32, C.POINTER(C.c_double), C.POINTER(C.c_double)]
     ops, mhz = C.c_double(), C.c_double()
-    _check(lib().gift_probe_pipe(device, kind, iters, C.byref(ops), C.byref(mhz)), "gift_probe_pipe")
+    rc = probe.gift_probe_pipe(device, kind, iters, C.byref(ops), C.byref(mhz))
+    if rc != 0:
+        raise RuntimeError("gift_probe_pipe failed (%d)" % rc)
     return ops.value, mhz.value
 
 
@@ -490,8 +540,15 @@ def gift_launch_count(ctx: Ctx) -> int:
     return ctx.launch_count()
 
 
+def gift_export_to_host(ctx: Ctx, *args, **kw):
+    ctx.export_to_host(*args, **kw)
+
+
+def gift_import_from_host(ctx: Ctx, *args, **kw):
+    ctx.import_from_host(*args, **kw)
+
+
 gift_resolve_args = resolve_args
 gift_slice_runs = slice_runs
-gift_probe_pipe = probe_pipe
 gift_strerror = strerror
 gift_version = version

@@ -6,8 +6,11 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libgift.so")
 HOSTCHECK = os.path.join(HERE, "libgift_hostcheck.so")
-SOURCES = ["gift_lib.cu", "gift_tokens.cu", "gift_order.cu", "gift_index.cu", "gift_chain.cu", "pipe_probe.cu"]
-HEADERS = ["gf128.cuh", "aes_tt.cuh", "gift_core.cuh", "gift_internal.cuh", "gift_rules.cuh", os.path.join("..", "..", "include", "gift.h")]
+PROBE = os.path.join(HERE, "libgift_probe.so")
+SOURCES = ["gift_lib.cu", "gift_rules.cu", "gift_hostio.cu", "gift_tokens.cu", "gift_order.cu", "gift_index.cu",
+           "gift_chain.cu"]
+HEADERS = ["gf128.cuh", "aes_tt.cuh", "gift_core.cuh", "gift_internal.cuh", "gift_rules.cuh", "gift_csr.cuh", "gift_seg.cuh",
+           os.path.join("..", "..", "include", "gift.h")]
 
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
               "-shared", "-Xcompiler", "-fPIC"]
@@ -37,6 +40,17 @@ def build_lib(force=False, verbose=False):
     return LIB
 
 
+def build_probe(force=False):
+    """Compile the instruction-rate probes (diagnostics, not part of libgift.so) for sm_100a."""
+    if not force and not _stale(PROBE, _deps(["pipe_probe.cu"])):
+        return PROBE
+    nvcc = os.environ.get("NVCC", "/usr/local/cuda/bin/nvcc")
+    tmp = PROBE + ".tmp.%d" % os.getpid()
+    subprocess.run([nvcc] + NVCC_FLAGS + ["-o", tmp, os.path.join(CSRC, "pipe_probe.cu")], check=True)
+    os.replace(tmp, PROBE)
+    return PROBE
+
+
 def build_hostcheck(force=False):
     """Compile the device arithmetic for the host (no GPU needed); returns the library path."""
     src = ["hostcheck.cpp"]
@@ -52,4 +66,5 @@ def build_hostcheck(force=False):
 
 if __name__ == "__main__":
     print(build_lib(force=True, verbose=True))
+    print(build_probe(force=True))
     print(build_hostcheck(force=True))

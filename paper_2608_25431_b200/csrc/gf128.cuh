@@ -66,37 +66,25 @@ GIFT_HD uint64_t mulwide(uint32_t a, uint32_t b)
     return (uint64_t)a * (uint64_t)b;
 }
 
-// Small multipliers (1, 2, 4, 128, 256) that the compiler cannot see through.  On this GPU
-// logic, permute and shift instructions share one pipe, which binds the cipher kernel,
-// while the multiply pipe is mostly idle.  An add written as a*1 + b, or a shift written
-// as a 32x32 -> 64 multiply by 2^s, stays a multiply instruction only if the factor is
-// not a compile-time constant; constant memory that the host could rewrite is opaque
-// enough.  The values never change.
+// A multiplier of 1 that the compiler cannot see through.  On this GPU logic, permute and
+// shift instructions share one pipe, which binds the cipher kernel, while the multiply pipe
+// is mostly idle.  An add written as a*1 + b stays a multiply-add instruction only if the
+// factor is not a compile-time constant; constant memory that the host could rewrite is
+// opaque enough.  The value never changes.
 #if defined(__CUDACC__)
-static __constant__ uint32_t gift_kmul[5] = {1u, 2u, 4u, 128u, 256u};
+static __constant__ uint32_t gift_kmul[1] = {1u};
 #endif
-static const uint32_t gift_kmul_host[5] = {1u, 2u, 4u, 128u, 256u};
+static const uint32_t gift_kmul_host[1] = {1u};
 #if defined(__CUDA_ARCH__)
 #define GIFT_KMUL(i) gift_kmul[i]
 #else
 #define GIFT_KMUL(i) gift_kmul_host[i]
 #endif
 
-#ifndef GIFT_ADD_ON_MUL
-#define GIFT_ADD_ON_MUL 1
-#endif
-#ifndef GIFT_REDUCE_ON_MUL
-#define GIFT_REDUCE_ON_MUL 0
-#endif
-
 // a + b on the multiply pipe
 GIFT_HD uint32_t add_mul(uint32_t a, uint32_t b)
 {
-#if GIFT_ADD_ON_MUL
     return a * GIFT_KMUL(0) + b;
-#else
-    return a + b;
-#endif
 }
 
 // Reverse the bits inside each byte of a little-endian word: block bytes <-> natural domain.
@@ -223,13 +211,11 @@ GIFT_HD void clmul128(const u128& a, const mulop& b, uint32_t r[8])
 }
 
 // Reduce a 256-bit polynomial modulo x^128 + x^7 + x^2 + x + 1: the high half h folds
-// down as h * (1 + x + x^2 + x^7).  Each shift of the 128-bit h by s bits is four
-// 32x32 -> 64 multiplies by 2^s (low word stays in place, high word carries into the next
-// word; the two never overlap, so they XOR straight into the sum).  The few bits pushed
-// past x^127 wrap around once more.
+// down as h * (1 + x + x^2 + x^7), every shifted copy built with funnel shifts across the
+// words; the few bits pushed past x^127 wrap around once more.  (Written with wide
+// multiplies by 2^s instead, the reduction spilled registers and was slower.)
 GIFT_HD u128 reduce256(const uint32_t r[8])
 {
-#if !GIFT_REDUCE_ON_MUL
     const uint32_t h0 = r[4], h1 = r[5], h2 = r[6], h3 = r[7];
     uint32_t t0 = h0 ^ (h0 << 1) ^ (h0 << 2) ^ (h0 << 7);
     uint32_t t1 = h1 ^ fshl(h0, h1, 1) ^ fshl(h0, h1, 2) ^ fshl(h0, h1, 7);
@@ -240,28 +226,6 @@ GIFT_HD u128 reduce256(const uint32_t r[8])
     u128 zz;
     zz.w[0] = r[0] ^ t0; zz.w[1] = r[1] ^ t1; zz.w[2] = r[2] ^ t2; zz.w[3] = r[3] ^ t3;
     return zz;
-#endif
-    const uint32_t k2 = GIFT_KMUL(1), k4 = GIFT_KMUL(2), k128 = GIFT_KMUL(3);
-    u128 z;
-    // word 0 waits for the wrapped bits; words 1..3 take the carries of the word below
-    uint64_t a1 = mulwide(r[4], k2), a2 = mulwide(r[4], k4), a7 = mulwide(r[4], k128);
-    const uint32_t z0 = r[0] ^ r[4] ^ (uint32_t)a1 ^ (uint32_t)a2 ^ (uint32_t)a7;
-    uint32_t c1 = (uint32_t)(a1 >> 32), c2 = (uint32_t)(a2 >> 32), c7 = (uint32_t)(a7 >> 32);
-#if defined(__CUDA_ARCH__)
-#pragma unroll
-#endif
-    for (int k = 1; k < 4; k++) {
-        a1 = mulwide(r[4 + k], k2);
-        a2 = mulwide(r[4 + k], k4);
-        a7 = mulwide(r[4 + k], k128);
-        z.w[k] = r[k] ^ r[4 + k] ^ (uint32_t)a1 ^ (uint32_t)a2 ^ (uint32_t)a7 ^ c1 ^ c2 ^ c7;
-        c1 = (uint32_t)(a1 >> 32);
-        c2 = (uint32_t)(a2 >> 32);
-        c7 = (uint32_t)(a7 >> 32);
-    }
-    const uint32_t o = c1 ^ c2 ^ c7;                 // at most 7 bits past x^127
-    z.w[0] = z0 ^ o ^ (o * k2) ^ (o * k4) ^ (o * k128);
-    return z;
 }
 
 GIFT_HD u128 gfmul(const u128& a, const mulop& b)

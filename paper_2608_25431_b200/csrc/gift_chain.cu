@@ -110,6 +110,12 @@ __device__ void stage_pointwise(const RuleArgs& r, uint32_t tid, uint32_t nthr)
 __device__ void stage_segreduce(const RuleArgs& r, uint32_t tid, uint32_t nthr)
 {
     const int lane = tid & 31;
+    if (__ldcg(r.table_bad) != 0u) {
+        // index arrays that are no valid CSR description: the launch as a whole is rejected
+        for (uint32_t j = tid; j < r.n_out; j += nthr) r.out[j] = GIFT_OWNER_CONFLICT;
+        if (tid == 0 && r.n_out) { r.viol[0] = r.n_out; r.viol[1] = 0u; }
+        return;
+    }
     for (uint32_t w = tid >> 5; w < r.n_seg; w += nthr >> 5) {
         const int32_t t0 = ld(r.seg_ptr + w), t1 = ld(r.seg_ptr + w + 1);
         const int32_t e0 = ld(r.src_ptr + w), e1 = ld(r.src_ptr + w + 1);
@@ -155,6 +161,14 @@ rule_chain_kernel(const __grid_constant__ ChainArgs a)
         a.r[tid].viol[0] = 0u;
         a.r[tid].viol[1] = 0xFFFFFFFFu;
     }
+    // the index arrays of the reduction rules are inputs of the chain, so all of them are
+    // checked up front (their flags are zero on entry and are put back to zero at the end)
+    for (uint32_t k = 0; k < a.n; k++) {
+        const RuleArgs& r = a.r[k];
+        if (r.kind != GIFT_RULE_SEGREDUCE) continue;
+        const bool bad = csr_tables_bad(r, tid, nthr);
+        if (__any_sync(0xFFFFFFFFu, bad) && (tid & 31) == 0) atomicOr(r.table_bad, 1u);
+    }
     cl.sync();
     for (uint32_t k = 0; k < a.n; k++) {
         const RuleArgs& r = a.r[k];
@@ -162,6 +176,7 @@ rule_chain_kernel(const __grid_constant__ ChainArgs a)
         else stage_pointwise(r, tid, nthr);
         cl.sync();
     }
+    if (tid < a.n) *a.r[tid].table_bad = 0u;
 }
 
 }  // namespace
@@ -179,6 +194,7 @@ extern "C" int gift_propagate_chain(gift_ctx* c, const gift_rule* rules, const i
     for (uint32_t k = 0; k < n_rules; k++) {
         const int rc = fill_rule_args(&rules[k], in_maps[k], outs[k], viol + 2 * k, a.r[k]);
         if (rc != GIFT_OK) return rc;
+        a.r[k].table_bad = c->d_rule_flags + k;
         // The chain takes no snapshot: an input that is read at other indices than the one
         // written (the gather source, the block-owner map) must not overlap the stage's output.
         const gift_rule& g = rules[k];

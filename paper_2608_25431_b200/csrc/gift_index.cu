@@ -1,5 +1,5 @@
 // Two-level ownership index (paper sec. 4.2) and the first three steps of a flow rule
-// (paper sec. 4.3, "Generating IFT rules").
+// (paper sec. 4.3, rule generation).
 //
 // Level 1 maps a base address to a tensor record (base, shape, element size and the
 // ownership-related dimensions "odim"); level 2 maps the subscripts of those dimensions to

@@ -6,11 +6,13 @@
 #include <string.h>
 
 #include "../../include/gift.h"
+#include "gift_csr.cuh"
 
 namespace gift {
 
 struct RuleArgs {
-    uint32_t kind, n_out, n_in, n_seg, n_in0, n_in1, param_mask;
+    uint32_t kind, n_out, n_in, n_seg, n_in0, n_in1, n_src, param_mask;
+    uint32_t* table_bad;            // SEGREDUCE: set to 1 before the rule runs if seg_ptr / src_ptr are malformed
     const int32_t* in[8];
     const int32_t* seg_ptr;
     const int32_t* src_ptr;
@@ -59,7 +61,7 @@ inline int fill_rule_args(const gift_rule* rule, const int32_t* const* in_maps, 
     if (rule->n_out && !out) return GIFT_E_INVAL;
     memset(&r, 0, sizeof(r));
     r.kind = rule->kind; r.n_out = rule->n_out; r.n_in = rule->n_in; r.n_seg = rule->n_seg;
-    r.n_in0 = rule->n_in0; r.n_in1 = rule->n_in1; r.param_mask = rule->param_mask;
+    r.n_in0 = rule->n_in0; r.n_in1 = rule->n_in1; r.n_src = rule->n_src; r.param_mask = rule->param_mask;
     r.seg_ptr = rule->seg_ptr; r.src_ptr = rule->src_ptr; r.src_idx = rule->src_idx; r.gather = rule->gather;
     r.out = out; r.viol = viol;
     uint32_t want_in = 1;
@@ -83,6 +85,24 @@ inline int fill_rule_args(const gift_rule* rule, const int32_t* const* in_maps, 
     }
     return GIFT_OK;
 }
+
+#if defined(__CUDACC__)
+// Every thread of the calling group checks its share of the pairs of both pointer arrays;
+// returns true if this thread saw a malformed pair.
+__device__ __forceinline__ bool csr_tables_bad(const RuleArgs& r, uint32_t tid, uint32_t nthr)
+{
+    bool bad = false;
+    if (r.n_seg == 0) {
+        if (tid == 0) bad = !csr_single_ok(r.seg_ptr[0], r.n_out) || !csr_single_ok(r.src_ptr[0], r.n_src);
+        return bad;
+    }
+    for (uint32_t k = tid; k < r.n_seg; k += nthr) {
+        bad |= !csr_pair_ok(r.seg_ptr[k], r.seg_ptr[k + 1], k == 0, k + 1 == r.n_seg, r.n_out);
+        bad |= !csr_pair_ok(r.src_ptr[k], r.src_ptr[k + 1], k == 0, k + 1 == r.n_seg, r.n_src);
+    }
+    return bad;
+}
+#endif
 
 inline bool ranges_overlap(const void* a, size_t na, const void* b, size_t nb)
 {

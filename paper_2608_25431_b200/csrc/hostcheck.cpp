@@ -12,6 +12,7 @@
 #include <vector>
 
 #include "gift_core.cuh"
+#include "gift_csr.cuh"
 
 using namespace gift;
 
@@ -186,4 +187,16 @@ void hc_segment(const uint8_t* key, const uint8_t* nonce12, const uint8_t* src, 
         seg_emulate<2>(key, nonce12, src, dst, table, page_bytes, origin, len, run_blocks, mode, tag16);
 }
 
-}  // extern "C"
+
+// 1 if ptr[0..n) is a valid CSR pointer array for `limit` indexed items, by the pair checks the
+// label kernels use.
+int hc_csr_ok(const int32_t* ptr, uint32_t n, uint32_t limit)
+{
+    if (n == 0) return 0;
+    if (n == 1) return csr_single_ok(ptr[0], limit) ? 1 : 0;
+    for (uint32_t k = 0; k + 1 < n; k++)
+        if (!csr_pair_ok(ptr[k], ptr[k + 1], k == 0, k + 2 == n, limit)) return 0;
+    return 1;
+}
+
+}

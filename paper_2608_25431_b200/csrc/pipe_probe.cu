@@ -5,10 +5,23 @@
 // 1024 threads per SM over long unrolled chains of one instruction kind (eight
 // independent chains per thread hide the latency), times the loop with the SM
 // cycle counter and reports lane-operations per SM clock.
+//
+// Diagnostics only: built into libgift_probe.so, not into libgift.so, and not declared in
+// the public header.  Entry point:
+//   int gift_probe_pipe(int device, int kind, uint32_t iters, double* lane_ops_per_clk_per_sm, double* sm_mhz)
+// kind: 0 three-input logic, 1 32x32+64 wide multiply-add, 2 byte permute, 3 conflict-free
+// shared-memory load, 4 funnel shift, 5 integer add, 6 logic and wide multiply interleaved,
+// 7 32-bit multiply-add, 8 logic and shared loads interleaved, 9-19 further kinds and
+// pairings, 20-32 instruction mixes like the cipher kernel's.  Returns 0, or a negative code
+// (-1 bad argument, -3 CUDA error).  Host call; allocates a few KB, synchronises.
 #include <cuda_runtime.h>
 #include <stdint.h>
 
-#include "../../include/gift.h"
+#define GIFT_OK 0
+#define GIFT_E_INVAL (-1)
+#define GIFT_E_NOMEM (-2)
+#define GIFT_E_CUDA (-3)
+#define GIFT_E_RANGE (-4)
 
 namespace {
 

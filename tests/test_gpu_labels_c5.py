@@ -76,6 +76,38 @@ def test_segreduce_matches_oracle_including_attack_and_uncovered_outputs(ctx):
     assert np.array_equal(out, ro) and np.array_equal(viol, rv) and rv[0] > head + tail
 
 
+def test_segreduce_with_malformed_index_arrays_rejects_the_launch(ctx):
+    """Pointer arrays that are no valid CSR description (decreasing, negative, past the end) must end as
+    CONFLICT on every output, never as a stray read or write; twice, with a good table in between."""
+    rng = np.random.default_rng(23)
+    n_out, n_req = 5000, 120
+    cuts = np.sort(rng.choice(np.arange(1, n_out), size=n_req - 1, replace=False))
+    seg_ptr = np.concatenate([[0], cuts, [n_out]]).astype(np.int32)
+    nb = rng.integers(0, 9, size=n_req)
+    src_ptr = np.concatenate([[0], np.cumsum(nb)]).astype(np.int32)
+    kv = rng.integers(0, 4, size=int(src_ptr[-1]) + 3).astype(np.int32)
+    src_idx = rng.integers(0, kv.size, size=int(src_ptr[-1])).astype(np.int32)
+    tok = rng.integers(0, 4, size=n_out).astype(np.int32)
+
+    def both(sp, srp):
+        out, viol = _rule(ctx, binding.RULE_SEGREDUCE, [tok, kv], n_out, seg_ptr=sp, src_ptr=srp, src_idx=src_idx)
+        ro, rv = L.propagate(L.SEGREDUCE, [tok, kv], n_out, seg_ptr=sp, src_ptr=srp, src_idx=src_idx)
+        assert np.array_equal(out, ro) and np.array_equal(viol, rv)
+        return rv
+
+    good = both(seg_ptr, src_ptr)
+    bad_tables = []
+    sp = seg_ptr.copy(); sp[40], sp[41] = sp[41], sp[40]; bad_tables.append((sp, src_ptr))           # decreasing pair
+    sp = seg_ptr.copy(); sp[-1] = n_out + 1000; bad_tables.append((sp, src_ptr))                     # past the outputs
+    sp = seg_ptr.copy(); sp[0] = -5; bad_tables.append((sp, src_ptr))                                # negative start
+    srp = src_ptr.copy(); srp[-1] += 7; bad_tables.append((seg_ptr, srp))                            # past src_idx
+    srp = src_ptr.copy(); srp[10] = 2**31 - 1; bad_tables.append((seg_ptr, srp))                     # a huge entry in the middle
+    for sp, srp in bad_tables:
+        rv = both(sp, srp)
+        assert rv.tolist() == [n_out, 0]
+        assert both(seg_ptr, src_ptr).tolist() == good.tolist()                                      # the flag does not stick
+
+
 def test_config5_rules_tamper_detection_and_reencrypt():
     w = W.config5(layers=2)
     x = w.extra

@@ -12,7 +12,9 @@ from gpu_harness import (dev, gpu_decrypt, gpu_encrypt, make_ctx, np_, oracle_de
 
 pytestmark = pytest.mark.gpu
 
-VARIANTS = [0, 0x21, 0x22, 0x41, 0x42, 0x441, 0x421, 0x341, 0x241]      # default, then (threads/256, tables, chains)
+# default (tables of up to 1024 segments run as one fused launch), two AES tables, and the
+# split form (plan / scan / cipher launches) forced for small tables too
+VARIANTS = [0, binding.CTX_TWO_TABLES, binding.CTX_SPLIT_LAUNCH, binding.CTX_TWO_TABLES | binding.CTX_SPLIT_LAUNCH]
 
 
 def _roundtrip_exact(w, flags=0, in_place=False):
@@ -51,7 +53,7 @@ def test_config1_tiny_round_trip(flags):
         _roundtrip_exact(W.config1(seed_salt=salt), flags)
 
 
-@pytest.mark.parametrize("flags", [0, 0x21])
+@pytest.mark.parametrize("flags", VARIANTS)
 def test_config2_decode_rows(flags):
     _roundtrip_exact(W.config2(), flags)
 
@@ -81,7 +83,7 @@ def test_lengths_ragged_and_empty():
     ids, keys = np.arange(5, dtype=np.int32), np.frombuffer(rng.bytes(80), dtype=np.uint8).reshape(5, 16)
     buf = np.frombuffer(rng.bytes(o + 64), dtype=np.uint8).copy()
     w = W.Workload("ragged", ids, keys, 5, buf, buf.size, segs)
-    for flags in (0, 0x21):
+    for flags in VARIANTS[:3]:
         _roundtrip_exact(w, flags)
 
 
@@ -99,8 +101,8 @@ def test_empty_call_and_argument_errors():
         ctx.set_keys(np.array([99], dtype=np.int32), np.zeros((1, 16), dtype=np.uint8))
     assert e.value.code == binding.E_RANGE
     with pytest.raises(binding.GiftError):
-        binding.Ctx(4, 0, 0x33)
-    assert binding.version() >= 100 and ctx.launch_count() > 0
+        binding.Ctx(4, 0, 0x40)                   # no such flag
+    assert binding.version() >= 200 and ctx.launch_count() > 0
     ctx.close()
 
 
@@ -146,7 +148,8 @@ def test_one_segment_beyond_2_pow_24_blocks_uses_the_top_power_level():
     ctx.close()
 
 
-def test_export_status_rules_match_oracle():
+@pytest.mark.parametrize("flags", [0, binding.CTX_SPLIT_LAUNCH])
+def test_export_status_rules_match_oracle(flags):
     w = W.config2(n_users=8, vocab=64)
     om = w.owner_map.copy()
     om[1], om[2], om[3], om[4] = 5, binding.OWNER_NONE, binding.OWNER_PARAM, binding.OWNER_CONFLICT
@@ -155,7 +158,7 @@ def test_export_status_rules_match_oracle():
     segs["len"][6] = w.buf.size
     segs["flags"][0] = 0
     ids, keys = w.user_ids[:7], w.keys[:7]
-    ctx = make_ctx(w, user_ids=ids, keys=keys)
+    ctx = make_ctx(w, flags, user_ids=ids, keys=keys)
     src = dev(w.buf)
     dst = torch.full_like(src, 0xEE)
     tags, st = gpu_encrypt(ctx, w, src, dst, segs=segs, owner_map=om)
@@ -176,7 +179,7 @@ def test_export_status_rules_match_oracle():
     victim = 1 if big != 1 else 2
     pt4[int(segs4["page0"][victim])] = len(pt4) + 5
     w4.page_table = pt4
-    ctx4 = make_ctx(w4)
+    ctx4 = make_ctx(w4, flags)
     src4 = dev(w4.buf)
     tags4, st4 = gpu_encrypt(ctx4, w4, src4, None, segs=segs4, owner_map=om4)
     ref4 = w4.buf.copy()
@@ -188,9 +191,10 @@ def test_export_status_rules_match_oracle():
     ctx4.close()
 
 
-def test_import_failures_zero_fill_and_unown():
+@pytest.mark.parametrize("flags", [0, binding.CTX_SPLIT_LAUNCH])
+def test_import_failures_zero_fill_and_unown(flags):
     w = W.config2(n_users=12, vocab=500)
-    ctx = make_ctx(w, user_ids=w.user_ids[:11], keys=w.keys[:11])       # user 11 has no key
+    ctx = make_ctx(w, flags, user_ids=w.user_ids[:11], keys=w.keys[:11])       # user 11 has no key
     ct = w.buf.copy()
     ref_tags, _ = oracle_encrypt(w, w.buf, ct, owner_map=None)
     bad_ct = ct.copy()
@@ -286,6 +290,11 @@ def test_bound_aad_matches_oracle_and_detects_a_changed_role():
         expect = gcm.seg_decrypt(ref, ref.copy(), w.segs, ref_tags, w.user_ids, w.keys, w.max_users, w.page_table,
                                  w.page_bytes, verify_only=True, aad=moved)
         assert np.array_equal(st_(st), expect) and expect[n // 2] == 1 and expect.sum() == 1
+        if n > 2:                                # a table longer than the bound array is refused before any launch
+            ctx.bind_aad(dev(aad[: n - 1].copy()))
+            with pytest.raises(binding.GiftError) as e:
+                gpu_encrypt(ctx, w, dev(w.buf))
+            assert e.value.code == binding.E_RANGE
         ctx.bind_aad(None)                       # unbound again: plain tags
         buf2 = dev(w.buf)
         tags2, _ = gpu_encrypt(ctx, w, buf2)

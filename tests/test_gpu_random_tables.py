@@ -36,7 +36,7 @@ def _random_workload(rng, paged, page_bytes):
         w = W.Workload("rand_paged", ids, keys, n_users, buf, buf.size, segs, page_table=table,
                        page_bytes=page_bytes, owner_map=om, unit_bytes=page_bytes)
     else:
-        unit = 64
+        unit = int(rng.choice([64, 256]))           # 256 and above: small tables take the fused launch
         offs, o = [], 0
         for n in lens:
             o = (o + unit - 1) // unit * unit            # unit-aligned starts: every unit has one owner
@@ -62,7 +62,8 @@ def test_random_tables_match_oracle(paged, page_bytes):
     for trial in range(6):
         w = _random_workload(rng, paged, page_bytes)
         have = w.user_ids[:-1] if len(w.user_ids) > 1 and trial % 2 else w.user_ids      # sometimes a missing key
-        ctx = make_ctx(w, user_ids=have, keys=w.keys[: len(have)])
+        flags = binding.CTX_SPLIT_LAUNCH if trial % 3 == 2 else 0          # mostly the fused single launch
+        ctx = make_ctx(w, flags, user_ids=have, keys=w.keys[: len(have)])
         buf = dev(w.buf)
         tags, st = gpu_encrypt(ctx, w, buf)
         ref = w.buf.copy()

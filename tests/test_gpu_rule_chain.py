@@ -96,6 +96,30 @@ def test_random_chains_with_in_place_stages_and_ragged_sizes(ctx):
         assert np.array_equal(viol, rviol), n
 
 
+def test_chain_with_a_malformed_reduction_table_rejects_that_rule_only(ctx):
+    rng = np.random.default_rng(78)
+    n = 3000
+    a = rng.integers(0, 3, size=n)
+    cuts = np.sort(rng.choice(np.arange(n + 1), size=41, replace=False))
+    src_ptr = np.arange(41) * 2
+    src_idx = rng.integers(0, n, size=80)
+    bad_cuts = cuts.copy()
+    bad_cuts[5], bad_cuts[6] = bad_cuts[6], bad_cuts[5]
+    for seg_ptr in (bad_cuts, cuts, bad_cuts, cuts):
+        maps = {"a": a, "t": np.zeros(n), "u": np.zeros(n)}
+        stages = [
+            (binding.RULE_IDENTITY, ["a"], "t", n, {}),
+            (binding.RULE_SEGREDUCE, ["t", "a"], "u", n, {"seg_ptr": seg_ptr, "src_ptr": src_ptr, "src_idx": src_idx}),
+            (binding.RULE_IDENTITY, ["u"], "t", n, {}),
+        ]
+        got, viol, ref, rviol = run_chain(ctx, stages, maps)
+        for k in maps:
+            assert np.array_equal(got[k], ref[k]), k
+        assert np.array_equal(viol, rviol)
+        if seg_ptr is bad_cuts:
+            assert viol[2] == n and viol[3] == 0 and (got["u"] == L.CONFLICT).all()
+
+
 def test_chain_argument_errors(ctx):
     m = dev(np.arange(64, dtype=np.int32))
     g = dev(np.arange(64, dtype=np.int32))

@@ -224,3 +224,28 @@ def test_static_work_split_tiles_every_segment_exactly(hc):
         else:
             nb = (rng.pareto(1.0, size=n) * 50).astype(np.int64)
         check(nb.astype(np.int64), rng.random(n) < 0.9, int(rng.choice([1, 7, 3552, 4736])))
+
+
+def test_csr_pointer_check_matches_oracle_reading(hc):
+    """The pair checks the label kernels apply to untrusted CSR pointer arrays accept exactly the
+    tables the oracle's reading accepts (hand cases, then random ones)."""
+    from oracle import labels as L
+    hc.hc_csr_ok.argtypes = [C.c_void_p, C.c_uint32, C.c_uint32]
+
+    def ok(ptr, limit):
+        a = np.asarray(ptr, dtype=np.int32)
+        return bool(hc.hc_csr_ok(_p(a), a.size, limit))
+
+    hand = [([0, 2, 5, 6], 6, True), ([0, 5, 2, 6], 6, False), ([0, 2, 5, 7], 6, False), ([-1, 2, 5, 6], 6, False),
+            ([0, 0, 0], 0, True), ([3], 3, True), ([4], 3, False), ([-1], 3, False), ([1, 1], 0, False),
+            ([0, 2**31 - 1, 5], 6, False), ([2, 3], 3, True)]
+    for ptr, limit, want in hand:
+        assert ok(ptr, limit) == want == L.csr_ok(ptr, limit), (ptr, limit)
+    rng = np.random.default_rng(91)
+    for _ in range(500):
+        n = int(rng.integers(1, 12))
+        limit = int(rng.integers(0, 30))
+        ptr = np.sort(rng.integers(0, limit + 1, size=n)).astype(np.int32)
+        if rng.random() < 0.5:
+            ptr[int(rng.integers(0, n))] = int(rng.integers(-3, limit + 4))
+        assert ok(ptr, limit) == L.csr_ok(ptr, limit), (ptr, limit)

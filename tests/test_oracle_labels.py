@@ -172,3 +172,25 @@ def test_swap_space_keeps_ownership_with_the_blocks():
     assert viol.tolist() == [0, 0xFFFFFFFF] and om.tolist() == [N, 0, N, N, 2, 0, 1, 1]
     viol = L.swap_in(om, [4, 9], np.array([1, 1], np.int32))      # onto a live block, and out of range
     assert viol.tolist() == [2, 0] and om[4] == C
+
+
+def test_segreduce_with_a_malformed_table_rejects_the_whole_launch():
+    """Hand-built: index arrays that are no valid CSR description make every output CONFLICT."""
+    in0 = np.array([1, 1, 2, 2, 2, 3], dtype=np.int32)
+    in1 = np.array([1, 2, 3], dtype=np.int32)
+    good = dict(seg_ptr=[0, 2, 5, 6], src_ptr=[0, 1, 2, 3], src_idx=[0, 1, 2])
+    out, viol = L.propagate(L.SEGREDUCE, [in0, in1], 6, **good)
+    assert out.tolist() == [1, 1, 2, 2, 2, 3] and viol.tolist() == [0, 0xFFFFFFFF]
+    all_conflict = [L.CONFLICT] * 6
+    for bad in (dict(good, seg_ptr=[0, 5, 2, 6]),            # decreasing: two requests would claim rows 2..4
+                dict(good, seg_ptr=[0, 2, 5, 7]),            # runs past the outputs
+                dict(good, seg_ptr=[-1, 2, 5, 6]),           # negative start
+                dict(good, src_ptr=[0, 1, 2, 4]),            # runs past src_idx
+                dict(good, src_ptr=[0, 2, 1, 3]),            # decreasing
+                dict(good, src_ptr=[-2, 1, 2, 3])):
+        out, viol = L.propagate(L.SEGREDUCE, [in0, in1], 6, **bad)
+        assert out.tolist() == all_conflict and viol.tolist() == [6, 0], bad
+    assert L.csr_ok([0, 0, 0], 0) and L.csr_ok([3], 3) and not L.csr_ok([4], 3) and not L.csr_ok([], 3)
+    # a valid table that leaves outputs uncovered is not malformed: only those outputs conflict
+    out, viol = L.propagate(L.SEGREDUCE, [in0, in1], 6, seg_ptr=[1, 2, 5], src_ptr=[0, 1, 2], src_idx=[0, 1])
+    assert out.tolist() == [L.CONFLICT, 1, 2, 2, 2, L.CONFLICT] and viol.tolist() == [2, 0]

@@ -193,3 +193,65 @@ def test_segment_aad_matches_openssl_and_binds_the_tag():
     moved[2, 0] ^= 1                                                 # presented in another role
     st = gcm.seg_decrypt(ct, ct.copy(), w.segs, tags, w.user_ids, w.keys, w.max_users, aad=moved)
     assert st.tolist() == [0, 0, 1, 0, 0, 0, 0, 0]
+
+
+def _seg_table(rows):
+    """rows: (owner, offset, len, page0)"""
+    t = np.zeros(len(rows), dtype=W.SEG_DTYPE)
+    for i, (owner, off, ln, page0) in enumerate(rows):
+        t[i]["owner"], t[i]["offset"], t[i]["len"], t[i]["page0"] = owner, off, ln, page0
+        t[i]["nonce"] = np.arange(12, dtype=np.uint8) + i
+    return t
+
+
+def test_overlap_definition_on_hand_built_tables():
+    """Which segments share bytes is written down by hand for every table below."""
+    # flat, 256-byte buffer
+    flat = _seg_table([
+        (0, 0, 32, 0),        # 0: [0, 32)    overlaps 1
+        (1, 16, 32, 0),       # 1: [16, 48)   overlaps 0 and 2
+        (2, 32, 48, 0),       # 2: [32, 80)   overlaps 1 and contains 3
+        (3, 48, 16, 0),       # 3: [48, 64)   inside 2
+        (0, 80, 16, 0),       # 4: [80, 96)   touches 2, shares no byte
+        (1, 96, 0, 0),        # 5: empty, at the start of 6: never overlaps
+        (2, 96, 20, 0),       # 6: [96, 116)  alone
+        (3, 100, 16, 0),      # 7: offset not a multiple of 16: bad descriptor, takes no part (would hit 6)
+        (0, 128, 40, 0),      # 8: [128, 168) identical to 9
+        (1, 128, 40, 0),      # 9
+        (2, 240, 32, 0),      # 10: runs past the buffer: bad descriptor
+        (3, 240, 16, 0),      # 11: [240, 256) alone (10 does not count)
+    ])
+    assert gcm.overlapping(flat, 256).tolist() == [1, 1, 1, 1, 0, 0, 0, 0, 1, 1, 0, 0]
+    # paged, 8 physical pages of 64 bytes; chains listed in the page table
+    table = np.array([0, 1,      # seg 0: pages 0, 1
+                      2, 1,      # seg 1: pages 2, 1   (page 1 shared with seg 0)
+                      3,         # seg 2: page 3       alone
+                      4, 4,      # seg 3: page 4 twice (overlaps itself)
+                      5, 6,      # seg 4: 70 bytes: page 5 and six bytes of page 6
+                      6,         # seg 5: page 6       (shares its first bytes with seg 4)
+                      7, 9,      # seg 6: page 9 does not exist: bad descriptor
+                      7], dtype=np.int32)   # seg 7: page 7 alone (seg 6 does not count)
+    paged = _seg_table([(0, 0, 128, 0), (1, 0, 100, 2), (2, 0, 64, 4), (3, 0, 128, 5), (0, 0, 70, 7),
+                        (1, 0, 10, 9), (2, 0, 128, 10), (3, 0, 5, 12)])
+    assert gcm.overlapping(paged, 8 * 64, table, 64).tolist() == [1, 1, 0, 1, 1, 1, 0, 0]
+
+
+def test_overlapping_segments_are_refused_untouched():
+    rng = np.random.default_rng(5)
+    ids = np.arange(4, dtype=np.int32)
+    keys = np.frombuffer(rng.bytes(64), dtype=np.uint8).reshape(4, 16)
+    segs = _seg_table([(0, 0, 32, 0), (1, 16, 32, 0), (2, 64, 32, 0), (3, 96, 16, 0)])
+    buf = np.frombuffer(rng.bytes(128), dtype=np.uint8).copy()
+    out = buf.copy()
+    tags, st = gcm.seg_encrypt(buf, out, segs, ids, keys, 4, check_overlap=True)
+    assert st.tolist() == [32, 32, 0, 0]
+    assert np.array_equal(out[:64], buf[:64]) and not tags[:2].any()          # refused: bytes as they were, tag zero
+    ct, tag = gcm.gcm_encrypt(keys[2], segs["nonce"][2], buf[64:96])
+    assert out[64:96].tobytes() == ct and tags[2].tobytes() == tag
+    # without the check the same table is taken as it comes (undefined mix, not tested); decrypt side:
+    om = np.full(8, 7, dtype=np.int32)
+    back = out.copy()
+    st = gcm.seg_decrypt(out, back, segs, tags, ids, keys, 4, owner_map=om, unit_bytes=16, check_overlap=True)
+    assert st.tolist() == [32, 32, 0, 0]
+    assert np.array_equal(back[:64], out[:64]) and np.array_equal(back[64:112], buf[64:112])
+    assert om.tolist() == [7, 7, 7, 7, 2, 2, 3, 7]                            # refused segments leave labels alone
