@@ -403,6 +403,11 @@ int gift_labels_swap_in(gift_ctx* ctx, int32_t* owner_map, uint32_t n_units, con
 /* Text for a GIFT_E_* code; never NULL. */
 const char* gift_strerror(int code);
 
+/* For a call that returned GIFT_E_CUDA or GIFT_E_NOMEM: the CUDA runtime's name for the
+ * error and where in the library it was met, as text; the last such failure of the calling
+ * thread ("" if none).  Never NULL. */
+const char* gift_last_error_detail(void);
+
 /* Library version, major*10000 + minor*100 + patch. */
 uint32_t gift_version(void);
 

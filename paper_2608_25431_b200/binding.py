@@ -28,14 +28,17 @@ EXPORTS = [
     "gift_propagate_labels", "gift_propagate_chain", "gift_tok_encrypt", "gift_tok_decrypt", "gift_check_launch_order",
     "gift_resolve_args", "gift_slice_runs", "gift_expand_owners", "gift_labels_swap_out", "gift_labels_swap_in",
     "gift_strerror", "gift_version", "gift_launch_count", "gift_timing_enable", "gift_timing_read",
-    "gift_export_to_host", "gift_import_from_host",
+    "gift_export_to_host", "gift_import_from_host", "gift_last_error_detail",
 ]
 
 
 class GiftError(RuntimeError):
     def __init__(self, code, where):
         self.code = code
-        super().__init__("%s failed: %s (%d)" % (where, strerror(code), code))
+        detail = ""
+        if code in (E_CUDA, E_NOMEM):
+            detail = ": " + lib().gift_last_error_detail().decode()
+        super().__init__("%s failed: %s (%d)%s" % (where, strerror(code), code, detail))
 
 
 class _Pages(C.Structure):
@@ -154,6 +157,7 @@ def lib():
         l.gift_tok_decrypt.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_uint32, C.c_uint64, C.c_void_p,
                                        C.c_void_p, C.c_void_p, C.c_void_p]
         l.gift_check_launch_order.argtypes = [C.c_void_p, C.POINTER(_Trace), C.c_void_p, C.c_void_p, C.c_void_p]
+        l.gift_last_error_detail.restype = C.c_char_p
         l.gift_strerror.restype = C.c_char_p
         l.gift_strerror.argtypes = [C.c_int]
         l.gift_version.restype = C.c_uint32
@@ -546,6 +550,10 @@ def gift_export_to_host(ctx: Ctx, *args, **kw):
 
 def gift_import_from_host(ctx: Ctx, *args, **kw):
     ctx.import_from_host(*args, **kw)
+
+
+def gift_last_error_detail() -> str:
+    return lib().gift_last_error_detail().decode()
 
 
 gift_resolve_args = resolve_args

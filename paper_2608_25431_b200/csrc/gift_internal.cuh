@@ -80,14 +80,28 @@ void gift_scratch_free(SegScratch* sc);
 
 #define MAX_TIMED 1024u
 
+// Where the last failing CUDA runtime call of this thread was, for gift_last_error_detail().
+void gift_note_cuda_error(cudaError_t e, const char* file, int line);
+
 #define CU_TRY(expr)                                   \
     do {                                               \
         cudaError_t e_ = (expr);                       \
         if (e_ != cudaSuccess) {                       \
+            gift_note_cuda_error(e_, __FILE__, __LINE__); \
             return e_ == cudaErrorMemoryAllocation ? GIFT_E_NOMEM : GIFT_E_CUDA; \
         }                                              \
     } while (0)
 
+
+// For clean-up paths that go on regardless: remember a failure, clear it, continue.
+#define CU_NOTE(expr)                                  \
+    do {                                               \
+        cudaError_t e_ = (expr);                       \
+        if (e_ != cudaSuccess) {                       \
+            gift_note_cuda_error(e_, __FILE__, __LINE__); \
+            (void)cudaGetLastError();                  \
+        }                                              \
+    } while (0)
 
 // Makes a device current for the duration of a call and restores the previous one.
 struct DeviceGuard {

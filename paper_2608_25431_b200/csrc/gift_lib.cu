@@ -17,6 +17,23 @@ using namespace gift;
 #include "gift_internal.cuh"
 #include "gift_seg.cuh"
 
+static thread_local char g_error_detail[384] = "";
+
+// Keeps the newest failure first and the one before it behind, so that an error met in a
+// clean-up path is still visible when a later call trips over it.
+void gift_note_cuda_error(cudaError_t e, const char* file, int line)
+{
+    const char* base = file;
+    for (const char* p = file; *p; p++)
+        if (*p == '/') base = p + 1;
+    char prev[160];
+    snprintf(prev, sizeof(prev), "%s", g_error_detail);
+    char* cut = strstr(prev, "; before that: ");
+    if (cut) *cut = 0;
+    snprintf(g_error_detail, sizeof(g_error_detail), "%s (%s) at %s:%d%s%s", cudaGetErrorName(e), cudaGetErrorString(e),
+             base, line, prev[0] ? "; before that: " : "", prev);
+}
+
 namespace {
 
 // ---------------------------------------------------------------------------
@@ -98,6 +115,7 @@ int launch_crypt(gift_ctx* c, const CallArgs& a, cudaStream_t st)
 int launch_overlap_check(gift_ctx* c, SegScratch* sc, const CallArgs& a, cudaStream_t st)
 {
     if (a.page_table == nullptr) {
+        if (a.nseg > 65536u) return GIFT_E_RANGE;                // all pairs: bounded
         overlap_flat_kernel<<<(a.nseg + OVL_TILE - 1) / OVL_TILE, OVL_TILE, 0, st>>>(a, sc->overlap);
         c->launches++;
         return GIFT_OK;
@@ -106,7 +124,7 @@ int launch_overlap_check(gift_ctx* c, SegScratch* sc, const CallArgs& a, cudaStr
     if (n_phys > ((uint64_t)1 << 28)) return GIFT_E_RANGE;
     if (n_phys > c->claim_cap) {
         CU_TRY(cudaDeviceSynchronize());
-        cudaFree(c->d_claim); cudaFree(c->d_rule_flags);
+        CU_NOTE(cudaFree(c->d_claim));
         c->d_claim = nullptr; c->claim_cap = 0;
         CU_TRY(cudaMalloc(&c->d_claim, (size_t)n_phys * sizeof(int32_t)));
         c->claim_cap = n_phys;
@@ -219,7 +237,11 @@ int gift_scratch_ensure(gift_ctx* c, SegScratch* sc, uint32_t nseg)
 
 void gift_scratch_free(SegScratch* sc)
 {
-    cudaFree(sc->wprefix); cudaFree(sc->acc); cudaFree(sc->ticket); cudaFree(sc->overlap); cudaFree(sc->glob);
+    CU_NOTE(cudaFree(sc->wprefix));
+    CU_NOTE(cudaFree(sc->acc));
+    CU_NOTE(cudaFree(sc->ticket));
+    CU_NOTE(cudaFree(sc->overlap));
+    CU_NOTE(cudaFree(sc->glob));
     memset(sc, 0, sizeof(*sc));
 }
 
@@ -281,6 +303,11 @@ int gift_ctx_create(gift_ctx** out, int device, uint32_t max_users, uint32_t fla
     if (cudaDeviceSynchronize() != cudaSuccess) return fail(GIFT_E_CUDA);
     rc = gift_scratch_ensure(c, &c->scratch, 1024);
     if (rc != GIFT_OK) return fail(rc);
+    const cudaError_t pending = cudaGetLastError();
+    if (pending != cudaSuccess) {
+        gift_note_cuda_error(pending, __FILE__, __LINE__);
+        return fail(GIFT_E_CUDA);
+    }
     *out = c;
     return GIFT_OK;
 }
@@ -290,31 +317,39 @@ int gift_ctx_destroy(gift_ctx* c)
     if (!c) return GIFT_E_INVAL;
     DeviceGuard g(c->device);
     if (g.ok) {
-        cudaDeviceSynchronize();
-        if (c->d_hot) cudaMemset(c->d_hot, 0, (size_t)c->max_users * sizeof(KeyHot));
-        if (c->d_pow) cudaMemset(c->d_pow, 0, (size_t)c->max_users * POW_LEVELS * 256 * sizeof(u128));
-        if (c->d_stage_keys) cudaMemset(c->d_stage_keys, 0, (size_t)c->stage_cap * 16);
-        cudaDeviceSynchronize();
-        cudaFree(c->d_t0); cudaFree(c->d_isbox); cudaFree(c->d_hot); cudaFree(c->d_pow);
+        CU_NOTE(cudaDeviceSynchronize());
+        if (c->d_hot) CU_NOTE(cudaMemset(c->d_hot, 0, (size_t)c->max_users * sizeof(KeyHot)));
+        if (c->d_pow) CU_NOTE(cudaMemset(c->d_pow, 0, (size_t)c->max_users * POW_LEVELS * 256 * sizeof(u128)));
+        if (c->d_stage_keys) CU_NOTE(cudaMemset(c->d_stage_keys, 0, (size_t)c->stage_cap * 16));
+        CU_NOTE(cudaDeviceSynchronize());
+        CU_NOTE(cudaFree(c->d_t0));
+        CU_NOTE(cudaFree(c->d_isbox));
+        CU_NOTE(cudaFree(c->d_hot));
+        CU_NOTE(cudaFree(c->d_pow));
         gift_scratch_free(&c->scratch);
-        cudaFree(c->d_claim); cudaFree(c->d_rule_flags);
+        CU_NOTE(cudaFree(c->d_claim));
+        CU_NOTE(cudaFree(c->d_rule_flags));
         if (c->io_ready) {
             for (int i = 0; i < GIFT_IO_STREAMS; i++) {
                 gift_scratch_free(&c->io_scratch[i]);
-                if (c->io_done[i]) cudaEventDestroy(c->io_done[i]);
-                if (c->io_stream[i]) cudaStreamDestroy(c->io_stream[i]);
+                if (c->io_done[i]) CU_NOTE(cudaEventDestroy(c->io_done[i]));
+                if (c->io_stream[i]) CU_NOTE(cudaStreamDestroy(c->io_stream[i]));
             }
-            if (c->io_start) cudaEventDestroy(c->io_start);
+            if (c->io_start) CU_NOTE(cudaEventDestroy(c->io_start));
         }
-        cudaFree(c->d_stage_ids); cudaFree(c->d_stage_keys); cudaFree(c->d_snapshot); cudaFree(c->d_next_sync);
+        CU_NOTE(cudaFree(c->d_stage_ids));
+        CU_NOTE(cudaFree(c->d_stage_keys));
+        CU_NOTE(cudaFree(c->d_snapshot));
+        CU_NOTE(cudaFree(c->d_next_sync));
         if (c->h_stage) {
             memset(c->h_stage, 0, (size_t)c->stage_cap * 20);
-            cudaFreeHost(c->h_stage);
+            CU_NOTE(cudaFreeHost(c->h_stage));
         }
         if (c->ev) {
-            for (uint32_t i = 0; i < 2 * MAX_TIMED; i++) cudaEventDestroy(c->ev[i]);
+            for (uint32_t i = 0; i < 2 * MAX_TIMED; i++) CU_NOTE(cudaEventDestroy(c->ev[i]));
             delete[] c->ev;
         }
+        CU_NOTE(cudaGetLastError());
     }
     delete c;
     return GIFT_OK;
@@ -474,6 +509,8 @@ const char* gift_strerror(int code)
     default: return "unknown error";
     }
 }
+
+const char* gift_last_error_detail(void) { return g_error_detail; }
 
 uint32_t gift_version(void) { return GIFT_VERSION; }
 

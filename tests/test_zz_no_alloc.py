@@ -147,3 +147,9 @@ def test_static_scratch_export_allocates_nothing_for_a_table_larger_than_any_bef
     assert np.array_equal(ref[0], want[0]) and np.array_equal(ref[1], want[1])
     ctx.close()
     ctx2.close()
+
+
+def test_no_cuda_call_of_the_library_failed_silently():
+    """Clean-up paths go on after a failing CUDA call but remember it; by the end of a run (this
+    file is collected last) nothing must have been remembered."""
+    assert binding.gift_last_error_detail() == ""
