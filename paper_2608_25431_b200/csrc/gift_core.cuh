@@ -48,6 +48,22 @@ GIFT_HD u128 mul_by_power(const u128& a, const u128* powtab, uint64_t e)
     return r;
 }
 
+// Ask for the table entries that mul_by_power(.., e) will read, ahead of time (the exponent of
+// a lane's chain is known before its first block is hashed; the entries then arrive while the
+// rows are processed instead of sitting, one after the other, on the tail of the piece).
+GIFT_HD void pow_prefetch(const u128* powtab, uint64_t e)
+{
+#if defined(__CUDA_ARCH__)
+#pragma unroll
+    for (int m = 0; m < POW_LEVELS; m++) {
+        const uint32_t d = (uint32_t)(e >> (8 * m)) & 0xFFu;
+        if (d) asm volatile("prefetch.global.L1 [%0];" ::"l"(powtab + m * 256 + d));
+    }
+#else
+    (void)powtab; (void)e;
+#endif
+}
+
 // ---- static work split --------------------------------------------------------------------
 //
 // The accepted segments' weights are laid end to end and resident warp w takes the weight
@@ -255,7 +271,7 @@ GIFT_HD u128 run_lane(const Tab& tb, const uint32_t* rk, const CtrPrefix& pre, c
 //    j-1 are independent, so the table lookups of the cipher and the multiplies and logic
 //    of the hash can interleave inside one warp;
 //  - the ragged last row (and a partial last block) goes through predicated code once.
-template <int MODE, class Tab>
+template <int MODE, bool PEEL, class Tab>
 GIFT_HD u128 run_lane_rows(const Tab& tb, const uint32_t* rk, const CtrPrefix& pre, const mulop& hs,
                            const u128* powtab, const uint8_t* src, uint8_t* dst, const SegAddr& addr,
                            uint64_t seg_nblk, uint64_t run_first, uint32_t run_n, uint32_t tail, int lane)
@@ -279,14 +295,50 @@ GIFT_HD u128 run_lane_rows(const Tab& tb, const uint32_t* rk, const CtrPrefix& p
     }
     uint64_t off = base + within + (uint64_t)lane * 16;     // this lane's block of the current row
 
+    {
+        // the exponent this lane's chain will need at the end (see below)
+        const uint32_t n_mine = rows + ((rows * 32 + (uint32_t)lane) < run_n ? 1u : 0u);
+        if (n_mine) pow_prefetch(powtab, seg_nblk - run_first - ((uint32_t)lane + (n_mine - 1) * 32) + 1);
+    }
     Block c_prev;
     c_prev.d[0] = c_prev.d[1] = c_prev.d[2] = c_prev.d[3] = 0;
     bool pending = false;
     CtrGroup grp;
     grp.grp = ~(ctr >> 8);                                  // forces the first set-up
     grp.c2[0] = grp.c2[1] = grp.c2[2] = grp.c2[3] = 0;
+    uint32_t j = 0;
+    if (PEEL && rows != 0) {
+        // The first row on its own, without the hash update of a previous row (which would
+        // multiply zero): worth it where a piece is a handful of rows, i.e. in small calls; in
+        // large ones the extra copy of the cipher code costs more than the multiply it saves.
+        const Block d = load_block(src + off);
+        Block c = d;
+        if (MODE != MODE_VERIFY) {
+            uint32_t ks[4];
+            ctr_group_setup(tb, rk, pre, ctr, grp);
+            ctr_keystream_grouped(tb, rk, pre, grp, ctr, ks);
+            Block o;
+            o.d[0] = d.d[0] ^ ks[0]; o.d[1] = d.d[1] ^ ks[1];
+            o.d[2] = d.d[2] ^ ks[2]; o.d[3] = d.d[3] ^ ks[3];
+            store_block(dst + off, o);
+            if (MODE == MODE_ENCRYPT) c = o;
+        }
+        c_prev = c;
+        pending = true;
+        ctr += 32;
+        off += 512;
+        if (--rows_in_page == 0) {
+            pidx++;
+            if (1 < rows || (uint64_t)rows * 32 < run_n) {
+                base = (uint64_t)(uint32_t)addr.table[addr.origin + pidx] * addr.page_bytes;
+                off = base + (uint64_t)lane * 16;
+            }
+            rows_in_page = (uint32_t)(addr.page_bytes >> 9);
+        }
+        j = 1;
+    }
 #pragma unroll 1
-    for (uint32_t j = 0; j < rows; j++) {
+    for (; j < rows; j++) {
         const Block d = load_block(src + off);
         Block c = d;
         if (MODE != MODE_VERIFY) {

@@ -10,10 +10,10 @@
 //                        keystream + XOR + GHASH; the warp whose report completes a segment
 //                        finishes its tag (no waiting, tickets only)
 //   or the fused form (tables of at most FUSED_MAX_SEGS segments: the rows of a decode step)
-//     1. crypt_kernel<FUSED>  every CTA recomputes the weights and their prefix sum in shared
-//                        memory (a few microseconds of redundant work instead of three kernel
-//                        boundaries), every warp checks the segments its slice touches itself,
-//
+//     1. crypt_kernel<FUSED>  every CTA reads the table into shared memory and recomputes the
+//                        weights and their prefix sum there (a microsecond of redundant
+//                        work instead of three kernel boundaries); every warp checks the
+//                        segments its slice touches itself
 //   followed, for decrypt, by
 //     4. fixup_kernel    zero-fills failed segments and marks their units unowned.
 //
@@ -281,18 +281,27 @@ struct SmemTab {
 };
 
 // Word index inside a 64 KiB chunk: x*64 + parity*32 + lane.  A thread writes four
-// consecutive lanes' copies of one entry with one 16-byte store.
+// consecutive lanes' copies of one entry with one 16-byte store; all its loads of the
+// 1 KiB source table go out before the first store, so that their latency is paid once.
 template <int NT>
 __device__ __forceinline__ void fill_tables(const uint32_t* __restrict__ t0)
 {
     uint4* tabs = reinterpret_cast<uint4*>(smem_raw);
     constexpr uint32_t quads = (NT == 4 ? 2u : 1u) * 4096u;
-#pragma unroll 4
-    for (uint32_t q = threadIdx.x; q < quads; q += blockDim.x) {
+    constexpr int per_thread = (int)((quads + CRYPT_THREADS - 1) / CRYPT_THREADS);
+    uint32_t v[per_thread];
+#pragma unroll
+    for (int k = 0; k < per_thread; k++) {
+        const uint32_t idx = ((uint32_t)threadIdx.x + (uint32_t)k * CRYPT_THREADS) * 4u;
+        v[k] = __ldg(t0 + ((idx >> 6) & 255u));
+    }
+#pragma unroll
+    for (int k = 0; k < per_thread; k++) {
+        const uint32_t q = (uint32_t)threadIdx.x + (uint32_t)k * CRYPT_THREADS;
         const uint32_t idx = q * 4u;
-        const uint32_t chunk = idx >> 14, x = (idx >> 6) & 255u, parity = (idx >> 5) & 1u;
-        const uint32_t v = rotl32(__ldg(t0 + x), 8 * (int)(chunk * 2 + parity));
-        tabs[q] = make_uint4(v, v, v, v);
+        const uint32_t chunk = idx >> 14, parity = (idx >> 5) & 1u;
+        const uint32_t r = rotl32(v[k], 8 * (int)(chunk * 2 + parity));
+        if (q < quads) tabs[q] = make_uint4(r, r, r, r);
     }
 }
 
@@ -323,14 +332,15 @@ struct Pending {
 // WRITE_OK: the status word of a segment whose tag is fine is written here (fused form: no
 // plan kernel has written it before).
 template <int MODE, bool WRITE_OK, class Tab>
-__device__ __noinline__ void finish_pending(const CallArgs& a, const Tab& tb, const Pending* pend, uint32_t n, int lane)
+__device__ __noinline__ void finish_pending(const CallArgs& a, const gift_seg* segtab, const Tab& tb, const Pending* pend,
+                                            uint32_t n, int lane)
 {
     bool ok = false;
     uint32_t s = 0;
     if ((uint32_t)lane < n) {
         s = pend->seg[lane];
         const uint4 sv = pend->sum[lane];
-        const gift_seg seg = a.segs[s];
+        const gift_seg seg = segtab[s];
         const KeyHot* hk = a.hot + seg.owner;
         u128 sum;
         sum.w[0] = sv.x; sum.w[1] = sv.y; sum.w[2] = sv.z; sum.w[3] = sv.w;
@@ -366,7 +376,7 @@ __device__ __noinline__ void finish_pending(const CallArgs& a, const Tab& tb, co
             const int k = __ffs(m) - 1;
             m &= m - 1;
             const uint32_t sk = __shfl_sync(0xFFFFFFFFu, s, k);
-            const gift_seg seg = a.segs[sk];
+            const gift_seg seg = segtab[sk];
             uint64_t u0;
             const uint64_t nu = seg_unit_count(a, seg, &u0);
             for (uint64_t u = lane; u < nu; u += 32) a.owner_map[seg_unit(a, seg, u0, u)] = seg.owner;
@@ -374,24 +384,43 @@ __device__ __noinline__ void finish_pending(const CallArgs& a, const Tab& tb, co
     }
 }
 
-// Fused form, per CTA: the weights of all segments and their exclusive prefix sum in shared
-// memory (sp[0..nseg], sp[nseg] the total).  Only the descriptor checks that need no table
-// walk decide a weight here; what else can refuse a segment (a bad page entry, the labels, a
-// missing key, an overlap) is found by the warps whose slices touch it, which then skip it.
-// CTA 0 also writes the result of the segments refused here, which no slice touches.
+// Fused form, per CTA: the descriptors of all segments, their weights and the exclusive prefix
+// sum of the weights in shared memory (sseg[0..nseg), sp[0..nseg], sp[nseg] the total).  Only
+// the descriptor checks that need no table walk decide a weight here; what else can refuse
+// a segment (a bad page entry, the labels, a missing key, an overlap) is found by the warps
+// whose slices touch it, which then skip it.  CTA 0 also writes the result of the segments
+// refused here, which no slice touches.  Warp w takes the chunks of 32 segments w and
+// w + 24; the loads are issued first (fused_load) so that their latency hides behind the
+// table fill, the rest follows (fused_prefix).
+constexpr int FUSED_CHUNKS_PER_WARP = (FUSED_MAX_SEGS / 32 + CRYPT_THREADS / 32 - 1) / (CRYPT_THREADS / 32);
+
+__device__ __forceinline__ void fused_load(const CallArgs& a, gift_seg (&mine)[FUSED_CHUNKS_PER_WARP])
+{
+    const int lane = threadIdx.x & 31, wid = threadIdx.x >> 5;
+#pragma unroll
+    for (int q = 0; q < FUSED_CHUNKS_PER_WARP; q++) {
+        const uint32_t i = ((uint32_t)wid + (uint32_t)q * (CRYPT_THREADS / 32)) * 32u + (uint32_t)lane;
+        if (i < a.nseg) mine[q] = a.segs[i];
+    }
+}
+
 template <int MODE>
-__device__ __forceinline__ void fused_prefix(const CallArgs& a, unsigned long long* sp, unsigned long long* chunk_sums)
+__device__ __forceinline__ void fused_prefix(const CallArgs& a, const gift_seg (&mine)[FUSED_CHUNKS_PER_WARP], gift_seg* sseg,
+                                             unsigned long long* sp, unsigned long long* chunk_sums)
 {
     const int tid = threadIdx.x, lane = tid & 31, wid = tid >> 5;
     constexpr int NW = CRYPT_THREADS / 32;
     const uint32_t n_chunks = (a.nseg + 31u) >> 5;            // at most 32
-    for (uint32_t c = wid; c < n_chunks; c += NW) {
+#pragma unroll
+    for (int q = 0; q < FUSED_CHUNKS_PER_WARP; q++) {
+        const uint32_t c = (uint32_t)wid + (uint32_t)q * NW;
+        if (c >= n_chunks) break;                             // uniform across the warp
         const uint32_t i = c * 32u + (uint32_t)lane;
         unsigned long long w = 0ull;
         if (i < a.nseg) {
-            const gift_seg seg = a.segs[i];
-            if (!desc_bad_quick(a, seg)) {
-                w = seg_weight(seg_blocks(seg.len));
+            sseg[i] = mine[q];
+            if (!desc_bad_quick(a, mine[q])) {
+                w = seg_weight(seg_blocks(mine[q].len));
             } else if (blockIdx.x == 0) {
                 a.status[i] = GIFT_ST_BAD_DESC;
                 if (MODE == MODE_ENCRYPT) reinterpret_cast<uint4*>(a.tags)[i] = make_uint4(0u, 0u, 0u, 0u);
@@ -430,23 +459,29 @@ __global__ void __launch_bounds__(CRYPT_THREADS, 1) crypt_kernel(const __grid_co
     KeyHot* slot = reinterpret_cast<KeyHot*>(smem_raw + TAB_BYTES) + wid;
     Pending* pend = reinterpret_cast<Pending*>(smem_raw + TAB_BYTES + NW * sizeof(KeyHot)) + wid;
     unsigned long long* sp = reinterpret_cast<unsigned long long*>(smem_raw + TAB_BYTES + NW * (sizeof(KeyHot) + sizeof(Pending)));
+    gift_seg* sseg = reinterpret_cast<gift_seg*>(sp + FUSED_MAX_SEGS + 1 + 32);
     const unsigned long long* prefix = FUSED ? sp : a.wprefix;
+    const gift_seg* segtab = FUSED ? sseg : a.segs;
 
-    // the call's total weight and the slice of a warp (see scan_kernel)
+    // the call's total weight and the slice of a warp (see scan_kernel).  A CTA whose warps
+    // all lie past the work leaves as soon as it knows.
     uint64_t total_weight, slice;
     if (FUSED) {
-        fused_prefix<MODE>(a, sp, sp + FUSED_MAX_SEGS + 1);
+        gift_seg mine[FUSED_CHUNKS_PER_WARP];
+        fused_load(a, mine);
+        fill_tables<NT>(t0);                                 // no barrier needed before: disjoint shared memory
+        fused_prefix<MODE>(a, mine, sseg, sp, sp + FUSED_MAX_SEGS + 1);      // ends with a barrier
         total_weight = sp[a.nseg];
         slice = (total_weight + a.resident_warps - 1) / a.resident_warps;
         if (slice < MIN_SLICE) slice = MIN_SLICE;
+        if ((uint64_t)blockIdx.x * NW * slice >= total_weight) return;
     } else {
         total_weight = a.glob->total_weight;
         slice = a.glob->slice;
+        if ((uint64_t)blockIdx.x * NW * slice >= total_weight) return;
+        fill_tables<NT>(t0);
+        __syncthreads();
     }
-    // a CTA whose warps all lie past the work leaves before it fills its tables
-    if ((uint64_t)blockIdx.x * NW * slice >= total_weight) return;
-    fill_tables<NT>(t0);
-    __syncthreads();
     SmemTab<NT> tb;
     tb.lb0 = (uint32_t)lane * 4u;
     tb.lb1 = (uint32_t)lane * 4u + 128u;
@@ -479,7 +514,7 @@ __global__ void __launch_bounds__(CRYPT_THREADS, 1) crypt_kernel(const __grid_co
         if (p0 >= g1) break;
         const uint64_t p1 = prefix[s + 1];
         if (p1 == p0) continue;                                      // refused before the split: no weight
-        const gift_seg seg = a.segs[s];
+        const gift_seg seg = segtab[s];
         if (FUSED) {
             // every warp that holds a piece of the segment reaches the same verdict on its own;
             // the one that holds the segment's first weight unit writes it down
@@ -519,7 +554,7 @@ __global__ void __launch_bounds__(CRYPT_THREADS, 1) crypt_kernel(const __grid_co
             // overhead weight or its last partial row): nothing to read, only the report below
         } else if (a.page_table == nullptr || (a.page_bytes & 511) == 0) {
             // rows of 32 blocks never straddle a page: the pipelined row loop applies
-            part = run_lane_rows<MODE>(tb, rk, pre, slot->hs[0], a.pow + (size_t)seg.owner * (POW_LEVELS * 256),
+            part = run_lane_rows<MODE, FUSED>(tb, rk, pre, slot->hs[0], a.pow + (size_t)seg.owner * (POW_LEVELS * 256),
                                        a.src, a.dst, addr, nblk, run_first, run_n, (uint32_t)(seg.len & 15), lane);
         } else {
             part = run_lane<1, MODE>(tb, rk, pre, slot->hs[0], a.pow + (size_t)seg.owner * (POW_LEVELS * 256),
@@ -567,14 +602,14 @@ __global__ void __launch_bounds__(CRYPT_THREADS, 1) crypt_kernel(const __grid_co
             n_pend++;
             if (n_pend == 32u) {
                 __syncwarp();
-                finish_pending<MODE, FUSED>(a, tb, pend, n_pend, lane);
+                finish_pending<MODE, FUSED>(a, segtab, tb, pend, n_pend, lane);
                 __syncwarp();
                 n_pend = 0;
             }
         }
     }
     __syncwarp();
-    if (n_pend) finish_pending<MODE, FUSED>(a, tb, pend, n_pend, lane);
+    if (n_pend) finish_pending<MODE, FUSED>(a, segtab, tb, pend, n_pend, lane);
 }
 
 // Shared memory of one CTA of the cipher kernel.
@@ -582,7 +617,7 @@ template <int NT, bool FUSED>
 constexpr size_t crypt_smem_bytes()
 {
     return (NT == 4 ? 131072u : 65536u) + (CRYPT_THREADS / 32) * (sizeof(KeyHot) + sizeof(Pending)) +
-           (FUSED ? (FUSED_MAX_SEGS + 1 + 32) * sizeof(unsigned long long) : 0);
+           (FUSED ? (FUSED_MAX_SEGS + 1 + 32) * sizeof(unsigned long long) + FUSED_MAX_SEGS * sizeof(gift_seg) : 0);
 }
 
 // ---------------------------------------------------------------------------

@@ -118,7 +118,8 @@ void hc_slice_piece(uint64_t g0, uint64_t g1, uint64_t p0, uint64_t p1, uint64_t
 }  // extern "C"
 
 // One whole segment, decomposed exactly as the kernel does: runs of run_blocks
-// blocks, 32 lanes per run, U chains per lane.  mode: 0 encrypt, 1 decrypt, 2 verify.
+// blocks, 32 lanes per run, U chains per lane (U == 0: the row loop; U == 3: the row loop with
+// its first row peeled off, as small calls run it).  mode: 0 encrypt, 1 decrypt, 2 verify.
 // table == NULL: flat at byte offset origin; else paged from table entry origin.
 template <int U>
 static void seg_emulate(const uint8_t* key, const uint8_t* nonce12, const uint8_t* src, uint8_t* dst,
@@ -144,24 +145,34 @@ static void seg_emulate(const uint8_t* key, const uint8_t* nonce12, const uint8_
         const uint32_t n = (uint32_t)(nblk - first < run_blocks ? nblk - first : run_blocks);
         for (int lane = 0; lane < 32; lane++) {
             u128 c;
-            if (U == 0) {                 // the row-wise, software-pipelined loop (chains == 0 selects it)
+            if (U == 3) {
                 if (mode == 0)
-                    c = run_lane_rows<MODE_ENCRYPT>(tab(), hot.rk, pre, hot.hs[0], pow.data(), src, dst, addr,
+                    c = run_lane_rows<MODE_ENCRYPT, true>(tab(), hot.rk, pre, hot.hs[0], pow.data(), src, dst, addr,
+                                                   nblk, first, n, tail, lane);
+                else if (mode == 1)
+                    c = run_lane_rows<MODE_DECRYPT, true>(tab(), hot.rk, pre, hot.hs[0], pow.data(), src, dst, addr,
+                                                   nblk, first, n, tail, lane);
+                else
+                    c = run_lane_rows<MODE_VERIFY, true>(tab(), hot.rk, pre, hot.hs[0], pow.data(), src, dst, addr,
+                                                  nblk, first, n, tail, lane);
+            } else if (U == 0) {          // the row-wise, software-pipelined loop (chains == 0 selects it)
+                if (mode == 0)
+                    c = run_lane_rows<MODE_ENCRYPT, false>(tab(), hot.rk, pre, hot.hs[0], pow.data(), src, dst, addr,
                                                     nblk, first, n, tail, lane);
                 else if (mode == 1)
-                    c = run_lane_rows<MODE_DECRYPT>(tab(), hot.rk, pre, hot.hs[0], pow.data(), src, dst, addr,
+                    c = run_lane_rows<MODE_DECRYPT, false>(tab(), hot.rk, pre, hot.hs[0], pow.data(), src, dst, addr,
                                                     nblk, first, n, tail, lane);
                 else
-                    c = run_lane_rows<MODE_VERIFY>(tab(), hot.rk, pre, hot.hs[0], pow.data(), src, dst, addr,
+                    c = run_lane_rows<MODE_VERIFY, false>(tab(), hot.rk, pre, hot.hs[0], pow.data(), src, dst, addr,
                                                    nblk, first, n, tail, lane);
             } else if (mode == 0)
-                c = run_lane<(U ? U : 1), MODE_ENCRYPT>(tab(), hot.rk, pre, hot.hs[U ? U - 1 : 0], pow.data(), src, dst, addr,
+                c = run_lane<(U == 2 ? 2 : 1), MODE_ENCRYPT>(tab(), hot.rk, pre, hot.hs[U == 2 ? 1 : 0], pow.data(), src, dst, addr,
                                               nblk, first, n, tail, lane);
             else if (mode == 1)
-                c = run_lane<(U ? U : 1), MODE_DECRYPT>(tab(), hot.rk, pre, hot.hs[U ? U - 1 : 0], pow.data(), src, dst, addr,
+                c = run_lane<(U == 2 ? 2 : 1), MODE_DECRYPT>(tab(), hot.rk, pre, hot.hs[U == 2 ? 1 : 0], pow.data(), src, dst, addr,
                                               nblk, first, n, tail, lane);
             else
-                c = run_lane<(U ? U : 1), MODE_VERIFY>(tab(), hot.rk, pre, hot.hs[U ? U - 1 : 0], pow.data(), src, dst, addr,
+                c = run_lane<(U == 2 ? 2 : 1), MODE_VERIFY>(tab(), hot.rk, pre, hot.hs[U == 2 ? 1 : 0], pow.data(), src, dst, addr,
                                              nblk, first, n, tail, lane);
             s = xor128(s, c);
         }
@@ -183,8 +194,10 @@ void hc_segment(const uint8_t* key, const uint8_t* nonce12, const uint8_t* src, 
         seg_emulate<0>(key, nonce12, src, dst, table, page_bytes, origin, len, run_blocks, mode, tag16);
     else if (chains == 1)
         seg_emulate<1>(key, nonce12, src, dst, table, page_bytes, origin, len, run_blocks, mode, tag16);
-    else
+    else if (chains == 2)
         seg_emulate<2>(key, nonce12, src, dst, table, page_bytes, origin, len, run_blocks, mode, tag16);
+    else
+        seg_emulate<3>(key, nonce12, src, dst, table, page_bytes, origin, len, run_blocks, mode, tag16);
 }
 
 

@@ -109,7 +109,7 @@ def test_power_table_matches_square_and_multiply(hc):
         assert o.tobytes() == power(e), e
 
 
-@pytest.mark.parametrize("chains", [0, 1, 2])
+@pytest.mark.parametrize("chains", [0, 1, 2, 3])      # 0: row loop, 1-2: chains per lane, 3: row loop with the first row peeled
 def test_run_decomposition_reproduces_gcm(hc, chains):
     """Every (length, run length) split of a segment into runs, lanes and chains gives the oracle's bytes and tag."""
     rng = np.random.default_rng(3 + chains)
@@ -135,7 +135,7 @@ def test_run_decomposition_reproduces_gcm(hc, chains):
             assert tag3.tobytes() == ref_tag
 
 
-@pytest.mark.parametrize("pb,chains", [(160, 2), (160, 1), (512, 0), (1024, 0), (1536, 0)])
+@pytest.mark.parametrize("pb,chains", [(160, 2), (160, 1), (512, 0), (1024, 0), (1536, 0), (512, 3), (1536, 3)])
 def test_paged_addressing_reproduces_gcm(hc, pb, chains):
     rng = np.random.default_rng(9)
     for n in [100, 160, 161, 1000, 3000, 3200, 5 * pb, 5 * pb + 1, 7 * pb - 1]:
