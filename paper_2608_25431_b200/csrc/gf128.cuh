@@ -8,12 +8,13 @@
 // field product is the ordinary polynomial product reduced modulo
 // x^128 + x^7 + x^2 + x + 1.
 //
-// A 32x32 -> 64 carry-less product is built from 16 ordinary integer multiplies
-// of operands masked to every fourth bit: with at most 8 ones per operand no
-// 4-bit slot can overflow, so the low bit of every slot is the XOR the
-// carry-less product wants.  The four products of one residue class are
-// combined with XOR (adding them could overflow a slot), then masked.
-// 128x128 uses two Karatsuba levels (9 such products).
+// A 32x32 -> 64 carry-less product is built from ordinary integer multiplies of
+// operands masked to every fourth bit: with at most 8 ones per operand no 4-bit
+// slot can overflow, so the low bit of every slot is the XOR the carry-less
+// product wants.  The low word of the product takes 16 such 32-bit multiplies;
+// the high word is obtained as the low word of the product of the bit-reversed
+// operands (16 more), never from the high word of a wide multiply (see
+// clmul32_low).  128x128 uses two Karatsuba levels (9 such leaves).
 #pragma once
 #include <stdint.h>
 
@@ -66,15 +67,15 @@ GIFT_HD uint64_t mulwide(uint32_t a, uint32_t b)
     return (uint64_t)a * (uint64_t)b;
 }
 
-// A multiplier of 1 that the compiler cannot see through.  On this GPU logic, permute and
+// Multipliers 1 and 2 that the compiler cannot see through.  On this GPU logic, permute and
 // shift instructions share one pipe, which binds the cipher kernel, while the multiply pipe
-// is mostly idle.  An add written as a*1 + b stays a multiply-add instruction only if the
-// factor is not a compile-time constant; constant memory that the host could rewrite is
-// opaque enough.  The value never changes.
+// has room.  An add written as a*1 + b, or a shift by one written as a*2, stays a multiply
+// instruction only if the factor is not a compile-time constant; constant memory that the
+// host could rewrite is opaque enough.  The values never change.
 #if defined(__CUDACC__)
-static __constant__ uint32_t gift_kmul[1] = {1u};
+static __constant__ uint32_t gift_kmul[2] = {1u, 2u};
 #endif
-static const uint32_t gift_kmul_host[1] = {1u};
+static const uint32_t gift_kmul_host[2] = {1u, 2u};
 #if defined(__CUDA_ARCH__)
 #define GIFT_KMUL(i) gift_kmul[i]
 #else
@@ -118,96 +119,112 @@ GIFT_HD u128 xor128(const u128& a, const u128& b)
 #define GIFT_M2 0x44444444u
 #define GIFT_M3 0x88888888u
 
-// One multiplier operand split for the masked-integer product: bm[j] = b & M_j.
-struct split32 {
-    uint32_t m[4];
+// One 32-bit leaf of a fixed multiplier, split for the masked-integer product in both bit
+// orders: f[j] = b & M_j and r[j] = rev32(b) & M_j.
+struct alignas(16) leaf_op {
+    uint32_t f[4];
+    uint32_t r[4];
 };
 
-GIFT_HD split32 split_word(uint32_t b)
+GIFT_HD leaf_op split_leaf(uint32_t b)
 {
-    split32 s;
-    s.m[0] = b & GIFT_M0;
-    s.m[1] = b & GIFT_M1;
-    s.m[2] = b & GIFT_M2;
-    s.m[3] = b & GIFT_M3;
+    const uint32_t rb = brev32(b);
+    leaf_op s;
+    s.f[0] = b & GIFT_M0; s.f[1] = b & GIFT_M1; s.f[2] = b & GIFT_M2; s.f[3] = b & GIFT_M3;
+    s.r[0] = rb & GIFT_M0; s.r[1] = rb & GIFT_M1; s.r[2] = rb & GIFT_M2; s.r[3] = rb & GIFT_M3;
     return s;
 }
 
-// 32x32 -> 64 carry-less product of a with a pre-split b.
-GIFT_HD uint64_t clmul32(uint32_t a, const split32& b)
+// Low 32 bits of the carry-less product of a with a pre-split b (bm[j] = b & M_j).
+//
+// Class r collects the products a_i * b_j with i + j == r (mod 4); bit 4k + r of their XOR
+// is the wanted coefficient.  Only the LOW word of every integer product is used (a plain
+// 32-bit multiply): reading the high word of a 32x32 -> 64 product costs this GPU two extra
+// issue slots per read, which the wide form paid 72 times per block.  In the low word a slot
+// k holds at most k + 1 <= 8 ones per product, so two products can be ADDED by the
+// multiplier itself without a slot running over (14 at most below the top slot, and what
+// the top slot carries out falls off bit 31); the two sums are then XORed and masked by one
+// logic instruction.  The four masked classes occupy disjoint bits and are merged by adds,
+// issued as multiply-adds to keep them off the logic pipe.
+GIFT_HD uint32_t clmul32_low(uint32_t a, const uint32_t bm[4])
 {
     const uint32_t a0 = a & GIFT_M0, a1 = a & GIFT_M1, a2 = a & GIFT_M2, a3 = a & GIFT_M3;
-    // class r collects the products a_i * b_j with i + j == r (mod 4).  The four masked
-    // classes occupy disjoint bits, so they are merged with integer adds, issued as
-    // multiply-adds to keep them off the logic pipe.  Each 32-bit half is merged on its
-    // own: no carry can cross.
-    uint64_t c = mulwide(a0, b.m[0]) ^ mulwide(a1, b.m[3]) ^ mulwide(a2, b.m[2]) ^ mulwide(a3, b.m[1]);
-    uint32_t lo = (uint32_t)c & GIFT_M0, hi = (uint32_t)(c >> 32) & GIFT_M0;
-    c = mulwide(a0, b.m[1]) ^ mulwide(a1, b.m[0]) ^ mulwide(a2, b.m[3]) ^ mulwide(a3, b.m[2]);
-    lo = add_mul((uint32_t)c & GIFT_M1, lo);
-    hi = add_mul((uint32_t)(c >> 32) & GIFT_M1, hi);
-    c = mulwide(a0, b.m[2]) ^ mulwide(a1, b.m[1]) ^ mulwide(a2, b.m[0]) ^ mulwide(a3, b.m[3]);
-    lo = add_mul((uint32_t)c & GIFT_M2, lo);
-    hi = add_mul((uint32_t)(c >> 32) & GIFT_M2, hi);
-    c = mulwide(a0, b.m[3]) ^ mulwide(a1, b.m[2]) ^ mulwide(a2, b.m[1]) ^ mulwide(a3, b.m[0]);
-    lo = add_mul((uint32_t)c & GIFT_M3, lo);
-    hi = add_mul((uint32_t)(c >> 32) & GIFT_M3, hi);
-    return ((uint64_t)hi << 32) | lo;
+    const uint32_t c0 = ((a0 * bm[0] + a1 * bm[3]) ^ (a2 * bm[2] + a3 * bm[1])) & GIFT_M0;
+    const uint32_t c1 = ((a0 * bm[1] + a1 * bm[0]) ^ (a2 * bm[3] + a3 * bm[2])) & GIFT_M1;
+    const uint32_t c2 = ((a0 * bm[2] + a1 * bm[1]) ^ (a2 * bm[0] + a3 * bm[3])) & GIFT_M2;
+    const uint32_t c3 = ((a0 * bm[3] + a1 * bm[2]) ^ (a2 * bm[1] + a3 * bm[0])) & GIFT_M3;
+    return add_mul(c3, add_mul(c2, add_mul(c1, c0)));
 }
 
-// A fixed multiplier prepared for repeated use: the nine Karatsuba leaf
-// operands of b, each split into its four masked classes (36 words).
+// A 64-bit carry-less product P = a (x) b is kept as two words: lo = P mod x^32 and hr, the
+// low word of rev32(a) (x) rev32(b).  Reversing all 63 bits of P gives that second product,
+// so the high word of P is  hi = rev32(hr << 1)  (see hi_from_rev): the high half comes from
+// a second low-word product instead of from the high word of a wide multiply.  XOR is linear
+// in both forms, so sums of products stay in this split form until the very end.
+GIFT_HD uint32_t hi_from_rev(uint32_t hr)
+{
+    return brev32(hr * GIFT_KMUL(1));
+}
+
+// A fixed multiplier prepared for repeated use: the nine Karatsuba leaf operands of b.
 //   leaves: b0, b1, b0^b1 | b2, b3, b2^b3 | b0^b2, b1^b3, b0^b1^b2^b3
 struct mulop {
-    split32 leaf[9];
+    leaf_op leaf[9];
 };
 
 GIFT_HD mulop prepare_mulop(const u128& b)
 {
     mulop p;
     const uint32_t b0 = b.w[0], b1 = b.w[1], b2 = b.w[2], b3 = b.w[3];
-    p.leaf[0] = split_word(b0);
-    p.leaf[1] = split_word(b1);
-    p.leaf[2] = split_word(b0 ^ b1);
-    p.leaf[3] = split_word(b2);
-    p.leaf[4] = split_word(b3);
-    p.leaf[5] = split_word(b2 ^ b3);
-    p.leaf[6] = split_word(b0 ^ b2);
-    p.leaf[7] = split_word(b1 ^ b3);
-    p.leaf[8] = split_word(b0 ^ b1 ^ b2 ^ b3);
+    p.leaf[0] = split_leaf(b0);
+    p.leaf[1] = split_leaf(b1);
+    p.leaf[2] = split_leaf(b0 ^ b1);
+    p.leaf[3] = split_leaf(b2);
+    p.leaf[4] = split_leaf(b3);
+    p.leaf[5] = split_leaf(b2 ^ b3);
+    p.leaf[6] = split_leaf(b0 ^ b2);
+    p.leaf[7] = split_leaf(b1 ^ b3);
+    p.leaf[8] = split_leaf(b0 ^ b1 ^ b2 ^ b3);
     return p;
 }
 
-// 64x64 -> 128 carry-less product (one Karatsuba level) of (x0,x1) with leaves l[0..2].
-GIFT_HD void clmul64(uint32_t x0, uint32_t x1, const split32* l, uint32_t r[4])
+// 64x64 -> 128 carry-less product (one Karatsuba level) of (x0,x1), given with its word-wise
+// bit reversals (rx0,rx1), with leaves l[0..2].  The result has words 0..3; n[k] is the part
+// of word k in natural bit order (k = 0..2) and r[k] the part still in reversed form
+// (k = 1..3): word k = n[k] ^ hi_from_rev(r[k]).
+GIFT_HD void clmul64(uint32_t x0, uint32_t x1, uint32_t rx0, uint32_t rx1, const leaf_op* l, uint32_t n[3], uint32_t r[4])
 {
-    const uint64_t p0 = clmul32(x0, l[0]);
-    const uint64_t p2 = clmul32(x1, l[1]);
-    const uint64_t pm = clmul32(x0 ^ x1, l[2]);
-    const uint64_t mid = pm ^ p0 ^ p2;
-    r[0] = (uint32_t)p0;
-    r[1] = (uint32_t)(p0 >> 32) ^ (uint32_t)mid;
-    r[2] = (uint32_t)p2 ^ (uint32_t)(mid >> 32);
-    r[3] = (uint32_t)(p2 >> 32);
+    const uint32_t p0l = clmul32_low(x0, l[0].f), p0r = clmul32_low(rx0, l[0].r);
+    const uint32_t p2l = clmul32_low(x1, l[1].f), p2r = clmul32_low(rx1, l[1].r);
+    const uint32_t pml = clmul32_low(x0 ^ x1, l[2].f), pmr = clmul32_low(rx0 ^ rx1, l[2].r);
+    n[0] = p0l;
+    n[1] = pml ^ p0l ^ p2l;       // low word of the middle term
+    n[2] = p2l;
+    r[0] = 0u;
+    r[1] = p0r;
+    r[2] = pmr ^ p0r ^ p2r;       // high word of the middle term
+    r[3] = p2r;
 }
 
 // 128x128 -> 256 carry-less product, unreduced.
-GIFT_HD void clmul128(const u128& a, const mulop& b, uint32_t r[8])
+GIFT_HD void clmul128(const u128& a, const mulop& b, uint32_t out[8])
 {
-    uint32_t z0[4], z2[4], zm[4];
-    clmul64(a.w[0], a.w[1], &b.leaf[0], z0);
-    clmul64(a.w[2], a.w[3], &b.leaf[3], z2);
-    clmul64(a.w[0] ^ a.w[2], a.w[1] ^ a.w[3], &b.leaf[6], zm);
-    const uint32_t m0 = zm[0] ^ z0[0] ^ z2[0], m1 = zm[1] ^ z0[1] ^ z2[1];
-    const uint32_t m2 = zm[2] ^ z0[2] ^ z2[2], m3 = zm[3] ^ z0[3] ^ z2[3];
-    r[0] = z0[0];
-    r[1] = z0[1];
-    r[2] = z0[2] ^ m0;
-    r[3] = z0[3] ^ m1;
-    r[4] = z2[0] ^ m2;
-    r[5] = z2[1] ^ m3;
-    r[6] = z2[2];
-    r[7] = z2[3];
+    const uint32_t ra0 = brev32(a.w[0]), ra1 = brev32(a.w[1]), ra2 = brev32(a.w[2]), ra3 = brev32(a.w[3]);
+    uint32_t z0n[3], z0r[4], z2n[3], z2r[4], zmn[3], zmr[4];
+    clmul64(a.w[0], a.w[1], ra0, ra1, &b.leaf[0], z0n, z0r);
+    clmul64(a.w[2], a.w[3], ra2, ra3, &b.leaf[3], z2n, z2r);
+    clmul64(a.w[0] ^ a.w[2], a.w[1] ^ a.w[3], ra0 ^ ra2, ra1 ^ ra3, &b.leaf[6], zmn, zmr);
+    // middle term m = zm ^ z0 ^ z2, word k of it lands in word k + 2 of the result
+    const uint32_t mn0 = zmn[0] ^ z0n[0] ^ z2n[0], mn1 = zmn[1] ^ z0n[1] ^ z2n[1], mn2 = zmn[2] ^ z0n[2] ^ z2n[2];
+    const uint32_t mr1 = zmr[1] ^ z0r[1] ^ z2r[1], mr2 = zmr[2] ^ z0r[2] ^ z2r[2], mr3 = zmr[3] ^ z0r[3] ^ z2r[3];
+    out[0] = z0n[0];
+    out[1] = z0n[1] ^ hi_from_rev(z0r[1]);
+    out[2] = z0n[2] ^ mn0 ^ hi_from_rev(z0r[2]);
+    out[3] = mn1 ^ hi_from_rev(z0r[3] ^ mr1);
+    out[4] = z2n[0] ^ mn2 ^ hi_from_rev(mr2);
+    out[5] = z2n[1] ^ hi_from_rev(z2r[1] ^ mr3);
+    out[6] = z2n[2] ^ hi_from_rev(z2r[2]);
+    out[7] = hi_from_rev(z2r[3]);
 }
 
 // Reduce a 256-bit polynomial modulo x^128 + x^7 + x^2 + x + 1: the high half h folds

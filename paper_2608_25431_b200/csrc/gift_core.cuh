@@ -24,13 +24,12 @@ namespace gift {
 enum { MODE_ENCRYPT = 0, MODE_DECRYPT = 1, MODE_VERIFY = 2 };
 
 constexpr int POW_LEVELS = 4;          // exponents up to 2^32 - 1
-constexpr int MAX_CHAINS = 2;
 
 // Per-user key material read by the hot loop.  512 bytes, 16-byte aligned fields.
 struct KeyHot {
     uint32_t rk[44];                   // AES-128 round keys, LE column words
     uint32_t h[4];                     // hash subkey H = E_K(0), natural domain
-    mulop hs[MAX_CHAINS];              // H^32 and H^64, prepared multipliers
+    mulop hs;                          // H^32, prepared multiplier (the stride of a lane's hash chain)
     uint32_t valid;                    // 1 when a key is installed
     uint32_t pad[7];
 };
@@ -440,9 +439,7 @@ GIFT_HD void derive_key_hot(const Tab& tb, const uint32_t key[4], KeyHot* out, u
     out->h[0] = h.w[0]; out->h[1] = h.w[1]; out->h[2] = h.w[2]; out->h[3] = h.w[3];
     u128 p = h;
     for (int k = 0; k < 5; k++) p = gfmul(p, p);       // H^32
-    out->hs[0] = prepare_mulop(p);
-    p = gfmul(p, p);                                   // H^64
-    out->hs[1] = prepare_mulop(p);
+    out->hs = prepare_mulop(p);
     out->valid = 1u;
     for (int k = 0; k < 7; k++) out->pad[k] = 0u;
     *h_out = h;

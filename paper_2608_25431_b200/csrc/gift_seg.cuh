@@ -554,10 +554,10 @@ __global__ void __launch_bounds__(CRYPT_THREADS, 1) crypt_kernel(const __grid_co
             // overhead weight or its last partial row): nothing to read, only the report below
         } else if (a.page_table == nullptr || (a.page_bytes & 511) == 0) {
             // rows of 32 blocks never straddle a page: the pipelined row loop applies
-            part = run_lane_rows<MODE, FUSED>(tb, rk, pre, slot->hs[0], a.pow + (size_t)seg.owner * (POW_LEVELS * 256),
+            part = run_lane_rows<MODE, FUSED>(tb, rk, pre, slot->hs, a.pow + (size_t)seg.owner * (POW_LEVELS * 256),
                                        a.src, a.dst, addr, nblk, run_first, run_n, (uint32_t)(seg.len & 15), lane);
         } else {
-            part = run_lane<1, MODE>(tb, rk, pre, slot->hs[0], a.pow + (size_t)seg.owner * (POW_LEVELS * 256),
+            part = run_lane<1, MODE>(tb, rk, pre, slot->hs, a.pow + (size_t)seg.owner * (POW_LEVELS * 256),
                                      a.src, a.dst, addr, nblk, run_first, run_n, (uint32_t)(seg.len & 15), lane);
         }
         u128 sum;

@@ -131,6 +131,9 @@ static void seg_emulate(const uint8_t* key, const uint8_t* nonce12, const uint8_
     KeyHot hot;
     u128 h;
     derive_key_hot(tab(), k, &hot, &h);
+    u128 p64 = h;
+    for (int i = 0; i < 6; i++) p64 = gfmul(p64, p64);
+    const mulop hs64 = prepare_mulop(p64);      // H^64: the stride of two chains per lane
     std::vector<u128> pow(POW_LEVELS * 256);
     for (int m = 0; m < POW_LEVELS; m++) build_pow_level(h, m, &pow[m * 256]);
     uint32_t nonce[3];
@@ -147,32 +150,32 @@ static void seg_emulate(const uint8_t* key, const uint8_t* nonce12, const uint8_
             u128 c;
             if (U == 3) {
                 if (mode == 0)
-                    c = run_lane_rows<MODE_ENCRYPT, true>(tab(), hot.rk, pre, hot.hs[0], pow.data(), src, dst, addr,
+                    c = run_lane_rows<MODE_ENCRYPT, true>(tab(), hot.rk, pre, hot.hs, pow.data(), src, dst, addr,
                                                    nblk, first, n, tail, lane);
                 else if (mode == 1)
-                    c = run_lane_rows<MODE_DECRYPT, true>(tab(), hot.rk, pre, hot.hs[0], pow.data(), src, dst, addr,
+                    c = run_lane_rows<MODE_DECRYPT, true>(tab(), hot.rk, pre, hot.hs, pow.data(), src, dst, addr,
                                                    nblk, first, n, tail, lane);
                 else
-                    c = run_lane_rows<MODE_VERIFY, true>(tab(), hot.rk, pre, hot.hs[0], pow.data(), src, dst, addr,
+                    c = run_lane_rows<MODE_VERIFY, true>(tab(), hot.rk, pre, hot.hs, pow.data(), src, dst, addr,
                                                   nblk, first, n, tail, lane);
             } else if (U == 0) {          // the row-wise, software-pipelined loop (chains == 0 selects it)
                 if (mode == 0)
-                    c = run_lane_rows<MODE_ENCRYPT, false>(tab(), hot.rk, pre, hot.hs[0], pow.data(), src, dst, addr,
+                    c = run_lane_rows<MODE_ENCRYPT, false>(tab(), hot.rk, pre, hot.hs, pow.data(), src, dst, addr,
                                                     nblk, first, n, tail, lane);
                 else if (mode == 1)
-                    c = run_lane_rows<MODE_DECRYPT, false>(tab(), hot.rk, pre, hot.hs[0], pow.data(), src, dst, addr,
+                    c = run_lane_rows<MODE_DECRYPT, false>(tab(), hot.rk, pre, hot.hs, pow.data(), src, dst, addr,
                                                     nblk, first, n, tail, lane);
                 else
-                    c = run_lane_rows<MODE_VERIFY, false>(tab(), hot.rk, pre, hot.hs[0], pow.data(), src, dst, addr,
+                    c = run_lane_rows<MODE_VERIFY, false>(tab(), hot.rk, pre, hot.hs, pow.data(), src, dst, addr,
                                                    nblk, first, n, tail, lane);
             } else if (mode == 0)
-                c = run_lane<(U == 2 ? 2 : 1), MODE_ENCRYPT>(tab(), hot.rk, pre, hot.hs[U == 2 ? 1 : 0], pow.data(), src, dst, addr,
+                c = run_lane<(U == 2 ? 2 : 1), MODE_ENCRYPT>(tab(), hot.rk, pre, (U == 2 ? hs64 : hot.hs), pow.data(), src, dst, addr,
                                               nblk, first, n, tail, lane);
             else if (mode == 1)
-                c = run_lane<(U == 2 ? 2 : 1), MODE_DECRYPT>(tab(), hot.rk, pre, hot.hs[U == 2 ? 1 : 0], pow.data(), src, dst, addr,
+                c = run_lane<(U == 2 ? 2 : 1), MODE_DECRYPT>(tab(), hot.rk, pre, (U == 2 ? hs64 : hot.hs), pow.data(), src, dst, addr,
                                               nblk, first, n, tail, lane);
             else
-                c = run_lane<(U == 2 ? 2 : 1), MODE_VERIFY>(tab(), hot.rk, pre, hot.hs[U == 2 ? 1 : 0], pow.data(), src, dst, addr,
+                c = run_lane<(U == 2 ? 2 : 1), MODE_VERIFY>(tab(), hot.rk, pre, (U == 2 ? hs64 : hot.hs), pow.data(), src, dst, addr,
                                              nblk, first, n, tail, lane);
             s = xor128(s, c);
         }
