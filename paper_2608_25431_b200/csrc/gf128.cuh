@@ -67,15 +67,15 @@ GIFT_HD uint64_t mulwide(uint32_t a, uint32_t b)
     return (uint64_t)a * (uint64_t)b;
 }
 
-// Multipliers 1 and 2 that the compiler cannot see through.  On this GPU logic, permute and
+// A multiplier of 1 that the compiler cannot see through.  On this GPU logic, permute and
 // shift instructions share one pipe, which binds the cipher kernel, while the multiply pipe
-// has room.  An add written as a*1 + b, or a shift by one written as a*2, stays a multiply
-// instruction only if the factor is not a compile-time constant; constant memory that the
-// host could rewrite is opaque enough.  The values never change.
+// has room.  An add written as a*1 + b stays a multiply-add instruction only if the factor
+// is not a compile-time constant; constant memory that the host could rewrite is opaque
+// enough.  The value never changes.
 #if defined(__CUDACC__)
-static __constant__ uint32_t gift_kmul[2] = {1u, 2u};
+static __constant__ uint32_t gift_kmul[1] = {1u};
 #endif
-static const uint32_t gift_kmul_host[2] = {1u, 2u};
+static const uint32_t gift_kmul_host[1] = {1u};
 #if defined(__CUDA_ARCH__)
 #define GIFT_KMUL(i) gift_kmul[i]
 #else
@@ -120,7 +120,7 @@ GIFT_HD u128 xor128(const u128& a, const u128& b)
 #define GIFT_M3 0x88888888u
 
 // One 32-bit leaf of a fixed multiplier, split for the masked-integer product in both bit
-// orders: f[j] = b & M_j and r[j] = rev32(b) & M_j.
+// orders: f[j] = b & M_j and r[j] = (rev32(b) << 1) & M_j.
 struct alignas(16) leaf_op {
     uint32_t f[4];
     uint32_t r[4];
@@ -128,7 +128,7 @@ struct alignas(16) leaf_op {
 
 GIFT_HD leaf_op split_leaf(uint32_t b)
 {
-    const uint32_t rb = brev32(b);
+    const uint32_t rb = brev32(b) << 1;      // the shift of hi_from_rev, taken here once per key
     leaf_op s;
     s.f[0] = b & GIFT_M0; s.f[1] = b & GIFT_M1; s.f[2] = b & GIFT_M2; s.f[3] = b & GIFT_M3;
     s.r[0] = rb & GIFT_M0; s.r[1] = rb & GIFT_M1; s.r[2] = rb & GIFT_M2; s.r[3] = rb & GIFT_M3;
@@ -157,13 +157,14 @@ GIFT_HD uint32_t clmul32_low(uint32_t a, const uint32_t bm[4])
 }
 
 // A 64-bit carry-less product P = a (x) b is kept as two words: lo = P mod x^32 and hr, the
-// low word of rev32(a) (x) rev32(b).  Reversing all 63 bits of P gives that second product,
-// so the high word of P is  hi = rev32(hr << 1)  (see hi_from_rev): the high half comes from
-// a second low-word product instead of from the high word of a wide multiply.  XOR is linear
-// in both forms, so sums of products stay in this split form until the very end.
+// low word of rev32(a) (x) (rev32(b) << 1).  Reversing all 63 bits of P gives
+// rev32(a) (x) rev32(b), whose low word shifted up by one is the high word of P read
+// backwards: hi = rev32(hr)  (see hi_from_rev).  The high half thus comes from a second
+// low-word product instead of from the high word of a wide multiply.  XOR is linear in both
+// forms, so sums of products stay in this split form until the very end.
 GIFT_HD uint32_t hi_from_rev(uint32_t hr)
 {
-    return brev32(hr * GIFT_KMUL(1));
+    return brev32(hr);
 }
 
 // A fixed multiplier prepared for repeated use: the nine Karatsuba leaf operands of b.
