@@ -39,20 +39,25 @@ UNIT = "GB/s"
 # AES-CTR with the first round hoisted, GHASH by masked integer multiplies with two Karatsuba
 # levels) was 660 logic-pipe operations, 144 wide multiplies and 150 shared-memory lookups.
 # Cheaper formulations were found since (one-instruction table addressing with four tables,
-# class merges as multiply-adds, round-2 constants cached per 256 counters), so the budget
-# was LOWERED, which raises the ceiling: the figures below are what the best formulation
-# known to this build needs on each pipe (they equal what the kernel executes, by ncu).
-# `roofline.frac` uses the lowered budget; `frac_first_budget` is kept for comparison.
-# DRAM bytes per payload byte of the cipher kernel, from the ncu capture summarised in
-# profiles/crypt_kernel_c3_2layers.md (dram__bytes_read.sum + dram__bytes_write.sum over the
-# payload of that launch); traffic grows in proportion to the payload.
+# round-2 constants cached per 256 counters, and a carry-less multiply that takes only the low
+# words of 32-bit products, in both bit orders, with pairs of products added inside the
+# multiplier), so the budget was LOWERED, which raises the ceilings: the figures below are what
+# the best formulation known to this build needs on each pipe (they equal what the kernel
+# executes, by ncu: profiles/crypt_kernel_c3_2layers.md).  With them the issue slots bind
+# (978 instructions at 128 lanes per clock) slightly before the logic pipe (453 at 64), so
+# `roofline.frac` is taken against the issue ceiling and `alu_frac` against the logic pipe;
+# `frac_first_budget` is kept for comparison.
+# DRAM bytes per payload byte of the cipher kernel, from the same ncu capture
+# (dram__bytes_read.sum + dram__bytes_write.sum over the payload of that launch); traffic grows
+# in proportion to the payload.
 NCU_DRAM_BYTES_PER_PAYLOAD_BYTE = 1.919
 
 FIRST_ALU_OPS_PER_BLOCK = 660
-ALU_OPS_PER_BLOCK = 483          # logic / permute / shift lane-operations (the binding pipe)
-MUL_OPS_PER_BLOCK = 230          # multiply-pipe lane-operations: 144 wide multiplies + multiply-adds
-LDS_OPS_PER_BLOCK = 176          # shared-memory lane-loads (table lookups, key material)
-ALL_OPS_PER_BLOCK = 901          # every issued lane-instruction
+ALU_OPS_PER_BLOCK = 453          # logic / permute / shift lane-operations
+MUL_OPS_PER_BLOCK = 328          # multiply-pipe lane-operations (32-bit multiply-adds)
+LDS_OPS_PER_BLOCK = 167          # shared-memory lane-loads (table lookups, key material) and the data load/store
+XU_OPS_PER_BLOCK = 15            # bit reversals
+ALL_OPS_PER_BLOCK = 978          # every issued lane-instruction
 
 
 def build_workload(name: str, layers: int):
@@ -346,35 +351,37 @@ class Bench:
 
 
 def roofline_of(w, kern_ms, clocks, sms, peaks):
-    """Roofline of the dominant kernel (the cipher kernel), which the integer pipes bind."""
+    """Roofline of the dominant kernel (the cipher kernel): integer instruction throughput binds."""
     payload, nseg = w.payload_bytes, len(w.segs)
     nblk = int(((w.segs["len"].astype(np.int64) + 15) // 16).sum())
     f_mhz = clocks["sm_mhz"] or 1965.0
     hbm_gbs = peaks.get("hbm_gbs", 6650.0)
-    r_alu, r_mul, r_lds, r_issue = 64.0, 64.0, 32.0, 128.0        # lane-ops per SM clock, measured with the pipe probes
+    # lane-operations per SM clock, measured with the pipe probes (profiles/pipe_rates_b200.md)
+    r_alu, r_mul, r_lds, r_xu, r_issue = 64.0, 64.0, 32.0, 16.0, 128.0
     f = f_mhz * 1e6
-    t_alu = ALU_OPS_PER_BLOCK * nblk / (sms * r_alu * f)
-    t_mul = MUL_OPS_PER_BLOCK * nblk / (sms * r_mul * f)
-    t_lds = LDS_OPS_PER_BLOCK * nblk / (sms * r_lds * f)
-    t_issue = ALL_OPS_PER_BLOCK * nblk / (sms * r_issue * f)
-    t_hbm = (2.0 * payload + 56.0 * nseg) / (hbm_gbs * 1e9)
-    t_roof = max(t_alu, t_mul, t_lds, t_issue, t_hbm)
-    return {"bound": "alu", "achieved": ALU_OPS_PER_BLOCK * nblk / (kern_ms * 1e-3) / 1e12,
-            "peak": sms * r_alu * f / 1e12, "unit": "Top/s",
-            "frac": t_roof / (kern_ms * 1e-3), "traffic": NCU_DRAM_BYTES_PER_PAYLOAD_BYTE * payload,
+    t = {"alu": ALU_OPS_PER_BLOCK * nblk / (sms * r_alu * f), "mul": MUL_OPS_PER_BLOCK * nblk / (sms * r_mul * f),
+         "lds": LDS_OPS_PER_BLOCK * nblk / (sms * r_lds * f), "xu": XU_OPS_PER_BLOCK * nblk / (sms * r_xu * f),
+         "issue": ALL_OPS_PER_BLOCK * nblk / (sms * r_issue * f),
+         "hbm": (2.0 * payload + 56.0 * nseg) / (hbm_gbs * 1e9)}
+    binding_resource = max(t, key=t.get)
+    t_roof = t[binding_resource]
+    kern_s = kern_ms * 1e-3
+    return {"bound": "alu", "resource": binding_resource,
+            "achieved": ALL_OPS_PER_BLOCK * nblk / kern_s / 1e12, "peak": sms * r_issue * f / 1e12, "unit": "Top/s",
+            "frac": t_roof / kern_s, "alu_frac": t["alu"] / kern_s,
+            "traffic": NCU_DRAM_BYTES_PER_PAYLOAD_BYTE * payload,
             "traffic_note": "bytes per launch: ncu DRAM bytes per payload byte on the 2-layer capture x this payload",
             "kernel": "crypt_kernel", "kernel_ms": kern_ms,
-            "kernel_payload_gbs": payload / (kern_ms * 1e-3) / 1e9,
-            "hbm_achieved_gbs": 2.0 * payload / (kern_ms * 1e-3) / 1e9,
-            "hbm_frac_of_measured": 2.0 * payload / (kern_ms * 1e-3) / 1e9 / hbm_gbs,
-            "ceilings_gbs": {"alu": payload / t_alu / 1e9, "mul": payload / t_mul / 1e9,
-                             "lds": payload / t_lds / 1e9, "issue": payload / t_issue / 1e9,
-                             "hbm": payload / t_hbm / 1e9},
-            "frac_first_budget": (FIRST_ALU_OPS_PER_BLOCK * nblk / (sms * r_alu * f)) / (kern_ms * 1e-3),
+            "kernel_payload_gbs": payload / kern_s / 1e9,
+            "hbm_achieved_gbs": 2.0 * payload / kern_s / 1e9,
+            "hbm_frac_of_measured": 2.0 * payload / kern_s / 1e9 / hbm_gbs,
+            "ceilings_gbs": {k: payload / v / 1e9 for k, v in t.items()},
+            "frac_first_budget": (FIRST_ALU_OPS_PER_BLOCK * nblk / (sms * r_alu * f)) / kern_s,
             "budget_per_block": {"alu": ALU_OPS_PER_BLOCK, "mul": MUL_OPS_PER_BLOCK, "lds": LDS_OPS_PER_BLOCK,
-                                 "all": ALL_OPS_PER_BLOCK, "first_alu": FIRST_ALU_OPS_PER_BLOCK},
+                                 "xu": XU_OPS_PER_BLOCK, "all": ALL_OPS_PER_BLOCK, "first_alu": FIRST_ALU_OPS_PER_BLOCK},
             "sm_mhz_used": f_mhz,
-            "peak_source": "148 SMs x 64 integer lanes x sampled SM clock; HBM from MEASURED_PEAKS.json (of measured)"
+            "peak_source": "achieved = issued lane-instructions per second, peak = 148 SMs x 4 schedulers x 32 lanes x sampled "
+                           "SM clock; HBM from MEASURED_PEAKS.json (of measured)"
             if peaks else "fallback HBM 6650 GB/s (of fallback)"}
 
 
@@ -662,7 +669,7 @@ def main():
                              name, b2.w.name, b2.nseg, b2.payload / 2**30, len(b2.w.user_ids), b2.layers),
                          "value": b2.payload * steps / (m2["total_ms"] * 1e-3) / 1e9, "unit": UNIT, "steps": steps,
                          "ms_per_step": m2["total_ms"] / steps, "kernel_ms": m2["kernel_ms"],
-                         "kernel_payload_gbs": r2["kernel_payload_gbs"], "frac": r2["frac"],
+                         "kernel_payload_gbs": r2["kernel_payload_gbs"], "frac": r2["frac"], "alu_frac": r2["alu_frac"],
                          "frac_first_budget": r2["frac_first_budget"], "clocks": m2["clocks"],
                          "gpu_launches": int(m2["launches"]),
                          "l2": "inputs larger than L2" if b2.flush is None else "L2 flushed before every step, outside its events"}

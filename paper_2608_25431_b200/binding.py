@@ -440,7 +440,8 @@ PROBE_KINDS = {0: "lop3", 1: "mad.wide.u32", 2: "prmt", 3: "ld.shared.u32", 4: "
                22: "lop3+prmt+mul.wide", 23: "3 lop3+ld.shared", 24: "2 lop3+mul.wide+ld.shared+xor",
                25: "2 lop3 (low half)+mul.wide", 26: "2 lop3 (high half)+mul.wide", 27: "2 lop3+mad.lo",
                28: "3 lop3+mul.wide", 29: "lop3(low,high)+lop3+mul.wide", 30: "mad.lo(high)+2 lop3+mul.wide",
-               31: "prmt(high)+lop3+mul.wide", 32: "mul.wide, 4 lop3, lop3(high)"}
+               31: "prmt(high)+lop3+mul.wide", 32: "mul.wide, 4 lop3, lop3(high)", 33: "brev", 34: "lop3+brev",
+               35: "mma.sync m16n8k128 b1 and.popc (one lane-op per thread)", 36: "2 mad.lo + lop3 on their results"}
 
 
 def probe_pipe(kind: int, iters: int = 2000, device: int = 0):

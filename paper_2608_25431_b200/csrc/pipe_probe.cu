@@ -12,7 +12,9 @@
 // kind: 0 three-input logic, 1 32x32+64 wide multiply-add, 2 byte permute, 3 conflict-free
 // shared-memory load, 4 funnel shift, 5 integer add, 6 logic and wide multiply interleaved,
 // 7 32-bit multiply-add, 8 logic and shared loads interleaved, 9-19 further kinds and
-// pairings, 20-32 instruction mixes like the cipher kernel's.  Returns 0, or a negative code
+// pairings, 20-32 instruction mixes like the first cipher kernel's, 33 bit reversal, 34 logic
+// and bit reversal, 35 the single-bit tensor-core product mma.sync m16n8k128 (and, popcount),
+// 36 two 32-bit multiply-adds feeding one logic operation.  Returns 0, or a negative code
 // (-1 bad argument, -3 CUDA error).  Host call; allocates a few KB, synchronises.
 #include <cuda_runtime.h>
 #include <stdint.h>
@@ -38,11 +40,12 @@ __global__ void __launch_bounds__(1024, 1) probe_kernel(uint32_t iters, uint32_t
     for (int i = threadIdx.x; i < 2048; i += blockDim.x) tab[i] = ((i >> 5) * 37u + seed) & 2047u & ~31u;
     __syncthreads();
     const volatile uint32_t* vtab = tab;
-    uint32_t x[CHAINS];
+    uint32_t x[CHAINS], y[CHAINS];
     unsigned long long w[CHAINS];
 #pragma unroll
     for (int c = 0; c < CHAINS; c++) {
         x[c] = seed * (c + 1) + threadIdx.x;
+        y[c] = seed + c;
         if (KIND == 3) x[c] = (x[c] & 2047u & ~31u);
         w[c] = x[c];
     }
@@ -179,6 +182,20 @@ __global__ void __launch_bounds__(1024, 1) probe_kernel(uint32_t iters, uint32_t
                     asm volatile("lop3.b32 %0, %0, %1, %2, 0x96;" : "+r"(x[c]) : "r"(k1), "r"(k1));
                     asm volatile("lop3.b32 %0, %0, %1, %2, 0x69;" : "+r"(x[c]) : "r"(k2), "r"(k2));
                     asm volatile("lop3.b32 %0, %0, %1, %2, 0x96;" : "+r"(x[c]) : "r"(k1), "r"((uint32_t)(w[c] >> 32)));
+                } else if (KIND == 33) {  // bit reversal
+                    asm volatile("brev.b32 %0, %0;" : "+r"(x[c]));
+                } else if (KIND == 34) {  // logic + bit reversal: separate pipes?
+                    asm volatile("lop3.b32 %0, %0, %1, %2, 0x96;" : "+r"(x[c]) : "r"(k1), "r"((uint32_t)w[c]));
+                    asm volatile("brev.b32 %0, %1;" : "=r"(*reinterpret_cast<uint32_t*>(&w[c])) : "r"(x[c]));
+                } else if (KIND == 35) {  // single-bit tensor-core product, 16x8x128 (and + popcount), counted as one lane-op per thread
+                    uint32_t* m = reinterpret_cast<uint32_t*>(&w[c]);
+                    asm volatile("mma.sync.aligned.m16n8k128.row.col.s32.b1.b1.s32.and.popc {%0,%1,%2,%3}, {%4,%5}, {%6}, {%0,%1,%2,%3};"
+                                 : "+r"(m[0]), "+r"(m[1]), "+r"(x[c]), "+r"(y[c]) : "r"(k1), "r"(k2), "r"(lane4));
+                } else if (KIND == 36) {  // two 32-bit multiply-adds whose sum feeds one logic operation (the shipped multiply's pattern)
+                    uint32_t* m = reinterpret_cast<uint32_t*>(&w[c]);
+                    asm volatile("mad.lo.u32 %0, %1, %2, %3;" : "=r"(m[0]) : "r"(x[c]), "r"(k1), "r"(m[1]));
+                    asm volatile("mad.lo.u32 %0, %1, %2, %3;" : "=r"(m[1]) : "r"(x[c]), "r"(k2), "r"(m[0]));
+                    asm volatile("lop3.b32 %0, %0, %1, %2, 0x96;" : "+r"(x[c]) : "r"(m[0]), "r"(m[1]));
                 } else if (KIND == 8) {   // logic and shared-memory loads interleaved
                     asm volatile("lop3.b32 %0, %0, %1, %2, 0x96;" : "+r"(x[c]) : "r"(k1), "r"(k2));
                     w[c] = vtab[lane4 + (c << 5)];
@@ -189,7 +206,7 @@ __global__ void __launch_bounds__(1024, 1) probe_kernel(uint32_t iters, uint32_t
     const long long t1 = clock64();
     uint32_t acc = 0;
 #pragma unroll
-    for (int c = 0; c < CHAINS; c++) acc ^= x[c] ^ (uint32_t)w[c] ^ (uint32_t)(w[c] >> 32);
+    for (int c = 0; c < CHAINS; c++) acc ^= x[c] ^ y[c] ^ (uint32_t)w[c] ^ (uint32_t)(w[c] >> 32);
     if (acc == 0x12345678u) sink[0] = acc;     // keeps the chains alive
     if (threadIdx.x == 0) cycles[blockIdx.x] = (unsigned long long)(t1 - t0);
 }
@@ -262,6 +279,10 @@ extern "C" int gift_probe_pipe(int device, int kind, uint32_t iters, double* lan
     case 30: e = run_probe<30>(sms, iters, d_cycles, d_sink, &ms); break;
     case 31: e = run_probe<31>(sms, iters, d_cycles, d_sink, &ms); break;
     case 32: e = run_probe<32>(sms, iters, d_cycles, d_sink, &ms); break;
+    case 33: e = run_probe<33>(sms, iters, d_cycles, d_sink, &ms); break;
+    case 34: e = run_probe<34>(sms, iters, d_cycles, d_sink, &ms); break;
+    case 35: e = run_probe<35>(sms, iters, d_cycles, d_sink, &ms); break;
+    case 36: e = run_probe<36>(sms, iters, d_cycles, d_sink, &ms); break;
     default: cudaFree(d_cycles); cudaFree(d_sink); cudaSetDevice(prev); return GIFT_E_INVAL;
     }
     int rc = GIFT_OK;
@@ -274,7 +295,8 @@ extern "C" int gift_probe_pipe(int device, int kind, uint32_t iters, double* lan
         for (int i = 0; i < sms; i++) mean += (double)h[i];
         mean /= sms;
         delete[] h;
-        static const double per_step[33] = {1, 1, 1, 1, 1, 1, 2, 1, 2, 1, 2, 2, 2, 2, 2, 3, 2, 2, 1, 2, 24, 3, 3, 4, 5, 3, 3, 3, 4, 3, 4, 3, 6};
+        static const double per_step[37] = {1, 1, 1, 1, 1, 1, 2, 1, 2, 1, 2, 2, 2, 2, 2, 3, 2, 2, 1, 2, 24, 3, 3, 4, 5, 3, 3, 3, 4, 3, 4, 3, 6,
+                                            1, 2, 1, 3};
         const double per_pair = per_step[kind];                       // instructions per step
         const double ops = 1024.0 * CHAINS * UNROLL * (double)iters * per_pair;
         *lane_ops_per_clk_per_sm = ops / mean;
