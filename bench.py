@@ -625,7 +625,7 @@ def main():
             line["e2e"] = {"value": e2e_value, "unit": UNIT,
                            "h2d_bytes_per_step": int(w.buf_bytes),
                            "d2h_bytes_per_step": int(w.buf_bytes + nseg * 20), "steps": k, "ms_per_step": e2e_ms,
-                           "mode": mode, "api": "gift_propagate_chain + gift_export_to_host",
+                           "mode": mode, "api": "the step's flow rules (gift_propagate_chain or gift_propagate_labels) + gift_export_to_host",
                            "launches_per_step": int(e2e_launches), "all_status_clear": ok_e2e}
             if slots is None:
                 # the opposite direction: upload ciphertext + tags, decrypt on the device, status words back
