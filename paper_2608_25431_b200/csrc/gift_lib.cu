@@ -83,13 +83,13 @@ __global__ void key_clear_kernel(const int32_t* __restrict__ ids, uint32_t n, Ke
 // host side of the segment calls
 // ---------------------------------------------------------------------------
 
-template <int MODE, int NT, bool FUSED>
+template <int MODE, int NT, bool FUSED, bool PEEL>
 int launch_crypt_t(gift_ctx* c, const CallArgs& a, cudaStream_t st)
 {
     constexpr size_t smem = crypt_smem_bytes<NT, FUSED>();
     constexpr int MAX_DEV = 64;
     static bool configured[MAX_DEV];
-    auto kern = crypt_kernel<MODE, NT, FUSED>;
+    auto kern = crypt_kernel<MODE, NT, FUSED, PEEL>;
     if (c->device < 0 || c->device >= MAX_DEV || !configured[c->device]) {
         CU_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
         if (c->device >= 0 && c->device < MAX_DEV) configured[c->device] = true;
@@ -105,10 +105,16 @@ int launch_crypt_t(gift_ctx* c, const CallArgs& a, cudaStream_t st)
     return GIFT_OK;
 }
 
-template <int MODE, bool FUSED>
-int launch_crypt(gift_ctx* c, const CallArgs& a, cudaStream_t st)
+// fused: the single-launch form (always with the first row peeled: its pieces are short).
+// short_segments: the table's segments are small on average, so pieces are short too.
+template <int MODE>
+int launch_crypt(gift_ctx* c, const CallArgs& a, cudaStream_t st, bool fused, bool short_segments)
 {
-    return c->tables == 4 ? launch_crypt_t<MODE, 4, FUSED>(c, a, st) : launch_crypt_t<MODE, 2, FUSED>(c, a, st);
+    if (fused)
+        return c->tables == 4 ? launch_crypt_t<MODE, 4, true, true>(c, a, st) : launch_crypt_t<MODE, 2, true, true>(c, a, st);
+    if (short_segments)
+        return c->tables == 4 ? launch_crypt_t<MODE, 4, false, true>(c, a, st) : launch_crypt_t<MODE, 2, false, true>(c, a, st);
+    return c->tables == 4 ? launch_crypt_t<MODE, 4, false, false>(c, a, st) : launch_crypt_t<MODE, 2, false, false>(c, a, st);
 }
 
 // The optional overlap check (GIFT_CTX_CHECK_OVERLAP): fills sc->overlap before the plan.
@@ -135,6 +141,8 @@ int launch_overlap_check(gift_ctx* c, SegScratch* sc, const CallArgs& a, cudaStr
     c->launches++;
     return GIFT_OK;
 }
+
+constexpr uint64_t SHORT_SEGMENT_BYTES = 4096;
 
 template <int MODE>
 int seg_call(gift_ctx* c, SegScratch* sc, const void* src, void* dst, uint64_t buf_bytes, const gift_seg* segs,
@@ -173,14 +181,19 @@ int seg_call(gift_ctx* c, SegScratch* sc, const void* src, void* dst, uint64_t b
     // stay with the split form, where that check runs once per segment.
     const bool cheap_labels = !labels || pages || MODE != MODE_ENCRYPT || labels->unit_bytes >= 256;
     if (allow_fused && nseg <= FUSED_MAX_SEGS && cheap_labels && !(c->flags & GIFT_CTX_SPLIT_LAUNCH)) {
-        rc = launch_crypt<MODE, true>(c, a, st);
+        rc = launch_crypt<MODE>(c, a, st, true, true);
         if (rc != GIFT_OK) return rc;
     } else {
         const uint32_t plan_blocks = (nseg + 7) / 8;          // 8 warps per block, one warp per segment
         plan_kernel<MODE><<<plan_blocks, 256, 0, st>>>(a);
         scan_kernel<<<1, 1024, 0, st>>>(a);
         c->launches += 2;
-        rc = launch_crypt<MODE, false>(c, a, st);
+        // Segments of one call do not overlap, so the buffer (or the page table) bounds their
+        // average size; where that bound is small the pieces are short and the kernel that peels
+        // their first row is the faster one.
+        uint64_t room = buf_bytes;
+        if (pages && (uint64_t)pages->n * pages->page_bytes < room) room = (uint64_t)pages->n * pages->page_bytes;
+        rc = launch_crypt<MODE>(c, a, st, false, room / nseg <= SHORT_SEGMENT_BYTES);
         if (rc != GIFT_OK) return rc;
     }
     if (MODE == MODE_DECRYPT) {

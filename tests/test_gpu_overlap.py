@@ -90,3 +90,39 @@ def test_without_the_flag_no_overlap_status_appears():
     _, st = gpu_encrypt(ctx, w, dev(w.buf), torch.zeros(w.buf.size, dtype=torch.uint8, device="cuda"))
     assert not (st_(st) & 32).any()
     ctx.close()
+
+
+def test_overlap_check_limits_and_the_static_entry():
+    """Flat tables beyond 65 536 segments are refused when the check is on; the allocation-free entry takes
+    flat tables with the check and refuses paged ones (their check needs memory that grows)."""
+    rng = np.random.default_rng(W.SEED_BASE + 460)
+    w = _flat_with_overlaps(rng, 300, 3)
+    ctx = make_ctx(w, binding.CTX_CHECK_OVERLAP)
+    src = dev(w.buf)
+    n = len(w.segs)
+    from gpu_harness import segs_dev
+    dst = torch.full_like(src, 0xEE)
+    tags = torch.zeros((n, 16), dtype=torch.uint8, device="cuda")
+    st = torch.zeros(n, dtype=torch.int32, device="cuda")
+    ctx.seg_encrypt_static(src, dst, segs_dev(w.segs), n, tags, st)
+    torch.cuda.synchronize()
+    ref = np.full_like(w.buf, 0xEE)
+    ref_tags, ref_st = gcm.seg_encrypt(w.buf, ref, w.segs, w.user_ids, w.keys, w.max_users, check_overlap=True)
+    assert np.array_equal(st_(st), ref_st) and np.array_equal(np_(tags), ref_tags) and np.array_equal(np_(dst), ref)
+    big_n = 65537
+    big = torch.zeros(40 * big_n, dtype=torch.uint8, device="cuda")
+    with pytest.raises(binding.GiftError) as e:
+        ctx.seg_encrypt(src, dst, big, big_n, torch.zeros((big_n, 16), dtype=torch.uint8, device="cuda"),
+                        torch.zeros(big_n, dtype=torch.int32, device="cuda"))
+    assert e.value.code == binding.E_RANGE
+    w4 = W.config4(total_bytes=4 << 20, cap_bytes=1 << 20, n_users=4)
+    ctx4 = make_ctx(w4, binding.CTX_CHECK_OVERLAP)
+    n4 = len(w4.segs)
+    with pytest.raises(binding.GiftError) as e:
+        ctx4.seg_encrypt_static(dev(w4.buf), dev(w4.buf), segs_dev(w4.segs), n4,
+                                torch.zeros((n4, 16), dtype=torch.uint8, device="cuda"),
+                                torch.zeros(n4, dtype=torch.int32, device="cuda"),
+                                page_table=dev(w4.page_table), page_bytes=w4.page_bytes)
+    assert e.value.code == binding.E_INVAL
+    ctx.close()
+    ctx4.close()

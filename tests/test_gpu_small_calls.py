@@ -134,3 +134,37 @@ def test_paged_small_table_with_bad_page_entries_and_labels():
     ctx = make_ctx(w)
     _check_export_and_import(ctx, w, rng)
     ctx.close()
+
+
+def test_many_short_segments_take_the_peeled_large_table_kernel():
+    """6 000 flat segments of at most 3 KiB in a buffer that leaves less than 4 KiB per segment: the
+    three-launch form with the kernel that peels the first row of every piece."""
+    rng = np.random.default_rng(W.SEED_BASE + 370)
+    nseg, n_users = 6000, 5
+    lens = rng.integers(0, 3073, size=nseg)
+    offs = np.concatenate([[0], np.cumsum((lens + 15) // 16 * 16)[:-1]])
+    segs = np.zeros(nseg, dtype=W.SEG_DTYPE)
+    segs["owner"] = rng.integers(0, n_users, size=nseg)
+    segs["offset"] = offs
+    segs["len"] = lens
+    segs["nonce"] = np.frombuffer(rng.bytes(12 * nseg), dtype=np.uint8).reshape(nseg, 12)
+    ids = np.arange(n_users, dtype=np.int32)
+    keys = np.frombuffer(rng.bytes(16 * n_users), dtype=np.uint8).reshape(n_users, 16).copy()
+    total = int(offs[-1]) + (int(lens[-1]) + 15) // 16 * 16 + 16
+    assert total // nseg <= 4096
+    buf = rng.integers(0, 256, size=total, dtype=np.uint8)
+    w = W.Workload("short", ids, keys, n_users, buf, buf.size, segs)
+    ctx = make_ctx(w)
+    d = dev(buf)
+    tags, st = gpu_encrypt(ctx, w, d)
+    ref = buf.copy()
+    ref_tags, ref_st = gcm.seg_encrypt(ref, ref, segs, ids, keys, n_users)
+    assert not ref_st.any() and not st_(st).any()
+    assert np.array_equal(np_(tags), ref_tags) and np.array_equal(np_(d), ref)
+    bad = ref.copy()
+    bad[int(offs[77]) + 3] ^= 2
+    st2 = gpu_decrypt(ctx, w, dev(bad), dev(ref_tags), verify_only=True)
+    assert st_(st2).sum() == 1 and st_(st2)[77] == 1
+    st3 = gpu_decrypt(ctx, w, d, tags)
+    assert not st_(st3).any() and np.array_equal(np_(d), buf)
+    ctx.close()
