@@ -57,6 +57,30 @@ int io_reserve(gift_ctx* c, const gift_chunk* chunks, uint32_t n_chunks)
     return GIFT_OK;
 }
 
+// The internal stream the next chunk goes to, made to wait for the caller's stream the first
+// time the call uses it.  With the overlap check of paged tables there is one claim array per
+// ctx, so every chunk then goes to the same stream.
+int io_slot(gift_ctx* c, bool used[GIFT_IO_STREAMS])
+{
+    const int slot = (c->flags & GIFT_CTX_CHECK_OVERLAP) ? 0 : (int)(c->io_next++ % GIFT_IO_STREAMS);
+    if (!used[slot]) {
+        if (cudaStreamWaitEvent(c->io_stream[slot], c->io_start, 0) != cudaSuccess) return -1;
+        used[slot] = true;
+    }
+    return slot;
+}
+
+// The caller's stream waits for every internal stream the call used.
+int io_join(gift_ctx* c, const bool used[GIFT_IO_STREAMS], cudaStream_t user)
+{
+    for (int i = 0; i < GIFT_IO_STREAMS; i++) {
+        if (!used[i]) continue;
+        CU_TRY(cudaEventRecord(c->io_done[i], c->io_stream[i]));
+        CU_TRY(cudaStreamWaitEvent(user, c->io_done[i], 0));
+    }
+    return GIFT_OK;
+}
+
 }  // namespace
 
 extern "C" int gift_export_to_host(gift_ctx* c, const void* h_src, void* h_dst, void* d_plain, void* d_cipher,
@@ -80,15 +104,11 @@ extern "C" int gift_export_to_host(gift_ctx* c, const void* h_src, void* h_dst, 
     cudaStream_t user = (cudaStream_t)stream;
     CU_TRY(cudaEventRecord(c->io_start, user));
     bool used[GIFT_IO_STREAMS] = {false, false, false};
-    for (uint32_t k = 0; k < n_chunks; k++) {
-        const gift_chunk& ch = chunks[k];
-        // the overlap check of paged tables keeps one claim array per ctx: one stream then
-        const int slot = (c->flags & GIFT_CTX_CHECK_OVERLAP) ? 0 : (int)(c->io_next++ % GIFT_IO_STREAMS);
+    // one chunk: upload, clear, encrypt out of place, download
+    auto enqueue = [&](const gift_chunk& ch) -> int {
+        const int slot = io_slot(c, used);
+        if (slot < 0) return GIFT_E_CUDA;
         cudaStream_t st = c->io_stream[slot];
-        if (!used[slot]) {
-            CU_TRY(cudaStreamWaitEvent(st, c->io_start, 0));
-            used[slot] = true;
-        }
         const uint64_t nb = ch.byte_hi - ch.byte_lo;
         const uint32_t ns = ch.seg_hi - ch.seg_lo;
         uint8_t* plain = (uint8_t*)d_plain + ch.byte_lo;
@@ -98,9 +118,9 @@ extern "C" int gift_export_to_host(gift_ctx* c, const void* h_src, void* h_dst, 
             CU_TRY(cudaMemsetAsync(cipher, 0, nb, st));
         }
         if (ns) {
-            rc = gift_seg_call_on(c, MODE_ENCRYPT, &c->io_scratch[slot], d_plain, d_cipher, buf_bytes, segs + ch.seg_lo,
-                                  ns, ch.seg_lo, pages, labels, d_tags + 16 * (size_t)ch.seg_lo, d_status + ch.seg_lo, st);
-            if (rc != GIFT_OK) return rc;
+            const int rc2 = gift_seg_call_on(c, MODE_ENCRYPT, &c->io_scratch[slot], d_plain, d_cipher, buf_bytes, segs + ch.seg_lo,
+                                             ns, ch.seg_lo, pages, labels, d_tags + 16 * (size_t)ch.seg_lo, d_status + ch.seg_lo, st);
+            if (rc2 != GIFT_OK) return rc2;
         }
         if (nb) CU_TRY(cudaMemcpyAsync((uint8_t*)h_dst + ch.byte_lo, cipher, nb, cudaMemcpyDeviceToHost, st));
         if (ns) {
@@ -108,13 +128,12 @@ extern "C" int gift_export_to_host(gift_ctx* c, const void* h_src, void* h_dst, 
                                    cudaMemcpyDeviceToHost, st));
             CU_TRY(cudaMemcpyAsync(h_status + ch.seg_lo, d_status + ch.seg_lo, (size_t)ns * 4, cudaMemcpyDeviceToHost, st));
         }
-    }
-    for (int i = 0; i < GIFT_IO_STREAMS; i++) {
-        if (!used[i]) continue;
-        CU_TRY(cudaEventRecord(c->io_done[i], c->io_stream[i]));
-        CU_TRY(cudaStreamWaitEvent(user, c->io_done[i], 0));
-    }
-    return GIFT_OK;
+        return GIFT_OK;
+    };
+    rc = GIFT_OK;
+    for (uint32_t k = 0; k < n_chunks && rc == GIFT_OK; k++) rc = enqueue(chunks[k]);
+    const int rc_join = io_join(c, used, user);       // also after a failure: what was enqueued must not outrun the caller's stream
+    return rc != GIFT_OK ? rc : rc_join;
 }
 
 extern "C" int gift_import_from_host(gift_ctx* c, const void* h_src, const uint8_t* h_tags, void* d_buf,
@@ -137,31 +156,26 @@ extern "C" int gift_import_from_host(gift_ctx* c, const void* h_src, const uint8
     cudaStream_t user = (cudaStream_t)stream;
     CU_TRY(cudaEventRecord(c->io_start, user));
     bool used[GIFT_IO_STREAMS] = {false, false, false};
-    for (uint32_t k = 0; k < n_chunks; k++) {
-        const gift_chunk& ch = chunks[k];
-        // the overlap check of paged tables keeps one claim array per ctx: one stream then
-        const int slot = (c->flags & GIFT_CTX_CHECK_OVERLAP) ? 0 : (int)(c->io_next++ % GIFT_IO_STREAMS);
+    // one chunk: upload ciphertext and tags, decrypt in place, status words back
+    auto enqueue = [&](const gift_chunk& ch) -> int {
+        const int slot = io_slot(c, used);
+        if (slot < 0) return GIFT_E_CUDA;
         cudaStream_t st = c->io_stream[slot];
-        if (!used[slot]) {
-            CU_TRY(cudaStreamWaitEvent(st, c->io_start, 0));
-            used[slot] = true;
-        }
         const uint64_t nb = ch.byte_hi - ch.byte_lo;
         const uint32_t ns = ch.seg_hi - ch.seg_lo;
         if (nb) CU_TRY(cudaMemcpyAsync((uint8_t*)d_buf + ch.byte_lo, (const uint8_t*)h_src + ch.byte_lo, nb, cudaMemcpyHostToDevice, st));
         if (ns) {
             CU_TRY(cudaMemcpyAsync(d_tags + 16 * (size_t)ch.seg_lo, h_tags + 16 * (size_t)ch.seg_lo, (size_t)ns * 16,
                                    cudaMemcpyHostToDevice, st));
-            rc = gift_seg_call_on(c, MODE_DECRYPT, &c->io_scratch[slot], d_buf, d_buf, buf_bytes, segs + ch.seg_lo, ns,
-                                  ch.seg_lo, pages, labels, d_tags + 16 * (size_t)ch.seg_lo, d_status + ch.seg_lo, st);
-            if (rc != GIFT_OK) return rc;
+            const int rc2 = gift_seg_call_on(c, MODE_DECRYPT, &c->io_scratch[slot], d_buf, d_buf, buf_bytes, segs + ch.seg_lo, ns,
+                                             ch.seg_lo, pages, labels, d_tags + 16 * (size_t)ch.seg_lo, d_status + ch.seg_lo, st);
+            if (rc2 != GIFT_OK) return rc2;
             CU_TRY(cudaMemcpyAsync(h_status + ch.seg_lo, d_status + ch.seg_lo, (size_t)ns * 4, cudaMemcpyDeviceToHost, st));
         }
-    }
-    for (int i = 0; i < GIFT_IO_STREAMS; i++) {
-        if (!used[i]) continue;
-        CU_TRY(cudaEventRecord(c->io_done[i], c->io_stream[i]));
-        CU_TRY(cudaStreamWaitEvent(user, c->io_done[i], 0));
-    }
-    return GIFT_OK;
+        return GIFT_OK;
+    };
+    rc = GIFT_OK;
+    for (uint32_t k = 0; k < n_chunks && rc == GIFT_OK; k++) rc = enqueue(chunks[k]);
+    const int rc_join = io_join(c, used, user);
+    return rc != GIFT_OK ? rc : rc_join;
 }

@@ -212,6 +212,7 @@ int seg_args_ok(gift_ctx* c, int mode, const void* src, void* dst, const gift_se
     *go = false;
     if (!c || !segs || !tags || !status) return nseg == 0 && c ? GIFT_OK : GIFT_E_INVAL;
     if (nseg == 0) return GIFT_OK;
+    if (nseg > (1u << 30)) return GIFT_E_RANGE;
     if (!src || (mode != MODE_VERIFY && !dst)) return GIFT_E_INVAL;
     if (((uintptr_t)src & 15) || ((uintptr_t)dst & 15) || ((uintptr_t)tags & 15)) return GIFT_E_ALIGN;
     if (pages && (!pages->table || pages->page_bytes == 0)) return GIFT_E_INVAL;
