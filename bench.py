@@ -346,6 +346,38 @@ class Bench:
         return {"total_ms": total_ms, "step_ms": step_ms, "kernel_ms": crypt_ms / max(1, crypt_n),
                 "kernel_launches": crypt_n, "clocks": clocks, "launches": self.ctx.launch_count() - l0}
 
+    def tamper_check(self):
+        """Config 5's seeded tampering at this size: 1 % of the segments get one ciphertext bit flipped,
+        one tag bit flipped, or another user as claimed owner; the import-side check must flag exactly
+        those (the other half of the metric: tamper-detect exactness).  Everything on the device."""
+        torch, w, x = self.torch, self.w, self.w.extra
+        self.ctx.seg_encrypt(self.buf, self.buf, self.segs, self.nseg, self.tags, self.status, **self.tables)
+        segs = w.segs.copy()
+        tags = self.tags.clone()
+        flips = []
+        for s_, kind, bit, tbit, wrong in zip(x["poisoned"], x["poison_kind"], x["poison_bit"], x["poison_tagbit"],
+                                             x["poison_owner"]):
+            s_ = int(s_)
+            if kind == 0:
+                flips.append((int(segs["offset"][s_]) + int(bit) // 8, 1 << (int(bit) % 8)))
+            elif kind == 1:
+                tags[s_, int(tbit) // 8] ^= 1 << (int(tbit) % 8)
+            else:
+                segs["owner"][s_] = int(wrong)
+        for addr, mask in flips:
+            self.buf[addr] ^= mask
+        d_segs = torch.from_numpy(segs.view(np.uint8).copy()).cuda()
+        st = torch.full((self.nseg,), 9, dtype=torch.int32, device="cuda")
+        self.ctx.verify_tags(self.buf, d_segs, self.nseg, tags, st)
+        torch.cuda.synchronize()
+        flagged = torch.nonzero(st != 0).flatten().cpu().numpy()
+        for addr, mask in flips:                      # put the ciphertext back
+            self.buf[addr] ^= mask
+        seeded = np.sort(np.asarray(x["poisoned"], dtype=np.int64))
+        return {"segments": int(self.nseg), "seeded": int(seeded.size), "flagged": int(flagged.size),
+                "exact": bool(np.array_equal(np.sort(flagged), seeded)),
+                "status_of_flagged": sorted(set(int(v) for v in st[st != 0].cpu().numpy().tolist()))}
+
     def close(self):
         self.ctx.close()
 
@@ -673,6 +705,8 @@ def main():
                          "frac_first_budget": r2["frac_first_budget"], "clocks": m2["clocks"],
                          "gpu_launches": int(m2["launches"]),
                          "l2": "inputs larger than L2" if b2.flush is None else "L2 flushed before every step, outside its events"}
+                if name == "c5":
+                    entry["tamper_detect"] = b2.tamper_check()
                 if name == "c2":
                     # the decode step's rows as a replayed CUDA graph (what a serving loop would do)
                     g2 = graph_of(b2.step)
