@@ -26,7 +26,8 @@
  *    so far (see gift_ctx_reserve) reallocates scratch, which synchronises.
  *  - gift_pages, gift_labels and gift_rule are small HOST structures that carry device
  *    pointers; they are read during the call and need not outlive it.
- *  - A ctx must not be used from two threads, or on two streams, at once.
+ *  - A ctx must not be used from two threads, or on two streams, at once (the
+ *    host-boundary calls say what they allow).
  *  - Ownership labels are int32: a user id >= 0, GIFT_OWNER_PARAM for model
  *    parameters (paper sec. 4.2 gives parameters an owner id of their own),
  *    GIFT_OWNER_NONE for memory no record covers (sec. 4.2, unowned memory may
@@ -154,11 +155,12 @@ int gift_clear_keys(gift_ctx* ctx, const int32_t* user_ids, uint32_t n, void* st
  * 16-byte GCM tag.  Otherwise the segment's dst bytes are left as they were,
  * its tag is 16 zero bytes and status[i] says why.  src may equal dst; bytes
  * outside all segments are never written.  Segments of one call must not
- * overlap (GIFT_CTX_CHECK_OVERLAP makes the call check it).  A table of at most 1024
- * segments runs as a single kernel launch.  buf_bytes is the size of src and of dst.  src and dst are addresses
- * the device can dereference: device memory, or page-locked host memory mapped
- * into the device's address space (the boundary copy of sec. 4.5 fused into
- * the cipher: the kernel then reads or writes across the bus itself). */
+ * overlap (GIFT_CTX_CHECK_OVERLAP makes the call check it).  A table of at most
+ * 1024 segments runs as a single kernel launch.  buf_bytes is the size of src
+ * and of dst.  src and dst are addresses the device can dereference: device
+ * memory, or page-locked host memory mapped into the device's address space
+ * (the boundary copy of sec. 4.5 fused into the cipher: the kernel then reads
+ * or writes across the bus itself). */
 int gift_seg_encrypt(gift_ctx* ctx, const void* src, void* dst, uint64_t buf_bytes,
                      const gift_seg* segs, uint32_t nseg, const gift_pages* pages,
                      const gift_labels* labels, uint8_t* tags_out, uint32_t* status, void* stream);
@@ -171,7 +173,7 @@ int gift_seg_encrypt(gift_ctx* ctx, const void* src, void* dst, uint64_t buf_byt
  * scratch with cudaMalloc when a call has more segments than any before it; this entry
  * point never does.  It calls no cudaMalloc, cudaFree or other allocating routine: its
  * scratch (work list, partial hashes, counters) is a fixed array inside the library image,
- * about 1.9 MB, which every GPU that loads the library holds until the process exits.
+ * about 2 MB, which every GPU that loads the library holds until the process exits.
  *   - Arguments, results and status words are exactly those of gift_seg_encrypt, bound AAD
  *     included; the ctx (created earlier, when allocation was still allowed) supplies the
  *     keys.  On a ctx with GIFT_CTX_CHECK_OVERLAP only flat tables are taken (the check of
@@ -206,7 +208,7 @@ int gift_ctx_bind_aad(gift_ctx* ctx, const uint8_t* aad16, uint32_t n);
  * are recorded as owned by the claimed owner.  On a mismatch, or when the
  * claimed owner has no key, the segment's dst bytes are all zero and the
  * covered units become GIFT_OWNER_NONE (a unit covered by both a good and a
- * failed segment ends up NONE).  BAD_DESC segments touch nothing. */
+ * failed segment ends up NONE).  BAD_DESC and OVERLAP segments touch nothing. */
 int gift_seg_decrypt(gift_ctx* ctx, const void* src, void* dst, uint64_t buf_bytes,
                      const gift_seg* segs, uint32_t nseg, const gift_pages* pages,
                      gift_labels* labels, const uint8_t* tags_in, uint32_t* status, void* stream);
@@ -432,7 +434,10 @@ int gift_timing_read(gift_ctx* ctx, double* total_ms, uint32_t* launches);
  * bus directions stay busy.  The work is ordered after what `stream` holds at the time of
  * the call, and `stream` waits for all of it; the call itself returns without waiting.
  * Copies are plain cudaMemcpyAsync, one per chunk and direction.  byte_lo and byte_hi are
- * multiples of 16. */
+ * multiples of 16.  Consecutive calls may be given different streams (and their own staging
+ * and host buffers) so that the download of one overlaps the upload of the next; they must
+ * still be issued from one thread.  With GIFT_CTX_CHECK_OVERLAP the check covers the segments
+ * of one chunk at a time, and all chunks run on one internal stream. */
 typedef struct {
     uint64_t byte_lo, byte_hi;
     uint32_t seg_lo, seg_hi;
